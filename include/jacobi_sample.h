@@ -1,0 +1,158 @@
+/*
+ * jacobi_sample.h - C ABI of the parallel autoregressive sampler for NVIDIA B200.
+ *
+ * The library draws samples x_1..x_T from a masked autoregressive network by
+ * solving the triangular system  x_t = h_t(u, x_{1:t-1}),  t = 1..T  (Eq. 1 and
+ * Eq. 5 of arXiv 2002.03629) with the random numbers u drawn beforehand by the
+ * caller (Appendix A.3).  Solvers: nonlinear Jacobi (Algorithm 1), Gauss-Seidel
+ * (Eq. 4; one sweep is the ordinary feedforward pass, Section 3.2) and the two
+ * block hybrids Jacobi-GS (Algorithm 2) and GS-Jacobi (Algorithm 3).  Every
+ * solver returns exactly the feedforward sample (Propositions 1 and 2).
+ *
+ * Conventions
+ *   - Pointers named *_dev are DEVICE pointers owned by the caller; pointers in
+ *     the model descriptors are HOST pointers, read during the create call only.
+ *   - Calls enqueue their work on `cuda_stream` (a cudaStream_t passed as
+ *     void*, NULL = default stream) and synchronise that stream before they
+ *     return, so outputs are complete and the return value is final.
+ *   - Return value: 0 = done and converged; JS_NOT_CONVERGED (1) = max_iters
+ *     reached while some sample still changed, outputs hold the last iterate;
+ *     negative = error, outputs unspecified.  No exceptions, no exit().
+ *   - One call at a time per model (the model owns the activation scratch).
+ *   - Positions are 0-based here (the paper counts from 1).  Symbols are bytes:
+ *     0/1 for binary positions, 0..C-1 for C-way positions.
+ *   - There is no CPU fallback: without a CUDA device every call fails with
+ *     JS_ERR_CUDA.
+ */
+#ifndef JACOBI_SAMPLE_H
+#define JACOBI_SAMPLE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct js_model js_model;   /* opaque; library-owned device memory */
+
+/* solver selection; block_hybrid(B) of the benchmark spec is JS_GS_JACOBI */
+typedef enum { JS_JACOBI = 0, JS_GAUSS_SEIDEL = 1, JS_GS_JACOBI = 2, JS_JACOBI_GS = 3 } js_mode;
+
+/* how u_t turns the conditional's logits z_t into x_t (Appendix A.3):
+ *   UNIFORM_ICDF  x = [u < sigmoid(z)]      noise [batch][T]      in (0,1)
+ *   LOGISTIC      x = [z + eps > 0]         noise [batch][T]      logistic
+ *   GUMBEL        x = argmax_c (z_c + g_c)  noise [batch][T][C]   Gumbel(0,1), lowest index wins ties */
+typedef enum { JS_NOISE_UNIFORM_ICDF = 0, JS_NOISE_LOGISTIC = 1, JS_NOISE_GUMBEL = 2 } js_noise_kind;
+typedef enum { JS_ACT_RELU = 0, JS_ACT_GELU_TANH = 1 } js_act;
+/* JS_F32: fp32 weights and activations.  JS_BF16: weights rounded to bf16 after
+ * masking, hidden activations rounded to bf16 after bias and nonlinearity,
+ * fp32 accumulation, fp32 logits. */
+typedef enum { JS_F32 = 0, JS_BF16 = 1 } js_prec;
+
+enum {
+    JS_OK = 0,
+    JS_NOT_CONVERGED = 1,
+    JS_ERR_ARG = -1,          /* null pointer, bad enum, batch > max_batch, ... */
+    JS_ERR_UNSUPPORTED = -2,  /* shape or mode the kernels do not cover */
+    JS_ERR_CUDA = -3,         /* a CUDA runtime call failed (js_last_cuda_error) */
+    JS_ERR_TIMEOUT = -4       /* a bounded device-side wait gave up; model stays usable */
+};
+
+/* Masked MLP (MADE).  Widths n = (T, H[0..L-1], T*C).  Input position d has
+ * degree d+1, output (d, c) has degree d+1, hidden unit j of a layer of width H
+ * has degree 1 + floor(j*(T-1)/H) unless hidden_deg gives it.  Hidden units read
+ * units of the layer below with degree <= their own, outputs read hidden units
+ * of strictly smaller degree, so position d depends on positions < d only.
+ * The library applies the masks and the rounding itself. */
+typedef struct {
+    int T;                         /* positions */
+    int C;                         /* logits per position: 1 = binary, else classes (<= 256) */
+    int L;                         /* hidden layers, 1..8 */
+    const int *H;                  /* [L] hidden widths */
+    int act;                       /* js_act */
+    int prec;                      /* js_prec */
+    const float *const *W;         /* [L+1] host pointers, W[l] unmasked [n[l+1]][n[l]] row-major */
+    const float *const *b;         /* [L+1] host pointers, b[l] [n[l+1]] */
+    const float *lut;              /* [n_lut] network input for symbol value v */
+    int n_lut;                     /* 2 for binary, C otherwise */
+    const int *const *hidden_deg;  /* NULL, or [L] host arrays of degrees (1..T-1) */
+    int max_batch;                 /* scratch is sized for this many samples */
+} js_made_desc;
+
+/* Masked-convolution stack (PixelCNN style): n_conv masked 3x3 convolutions
+ * with ReLU and zero padding, then a 1x1 head.  Image [height][width][in_ch],
+ * position t = (y*width + x)*in_ch + c.  Hidden channel k is in colour group
+ * floor(in_ch*k/ch).  Kernels keep the row above and the left neighbour; at the
+ * centre tap layer 0 keeps input groups < output group (type A), later layers
+ * groups <= (type B); the head gives sub-pixel c its C logits from groups <= c.
+ * W[0] [ch][3][3][in_ch], W[1..n_conv-1] [ch][3][3][ch], W[n_conv] [in_ch*C][ch]. */
+typedef struct {
+    int height, width, in_ch, ch, n_conv, C;
+    int prec;                      /* js_prec */
+    const float *const *W;         /* [n_conv+1] host pointers */
+    const float *const *b;         /* [n_conv+1] host pointers */
+    const float *lut;              /* [C] */
+    int n_lut;
+    int max_batch;
+} js_conv_desc;
+
+int js_made_create(const js_made_desc *desc, js_model **out);
+int js_conv_create(const js_conv_desc *desc, js_model **out);
+void js_model_destroy(js_model *m);
+
+/*
+ * Solve for all positions at once (Algorithms 1-3).
+ *   noise_dev        fp32, layout by `nk` above; the same values serve every iteration
+ *   init_dev         uint8 [batch][T] start iterate s^0, NULL = zeros; may alias out_samples_dev
+ *   mode, block      block = B, the number of consecutive positions per block, for the hybrids
+ *   max_iters        <= 0: the algorithm's own cap (T for Jacobi, |B_i| per block for
+ *                    GS-Jacobi, number of blocks for Jacobi-GS); otherwise that cap lowered
+ *   out_samples_dev  uint8 [batch][T]
+ *   out_iters_dev    int32 [batch] (may be NULL): iteration at which the sample's forward
+ *                    difference vanished, the confirming iteration included, or the cap;
+ *                    GS-Jacobi: summed over blocks; Jacobi-GS: outer iterations; Gauss-Seidel: 1
+ * A sample whose iterate did not change in an iteration is at its fixed point and stops
+ * counting; the call ends when every sample has stopped or the cap is reached.
+ */
+int jacobi_sample(const js_model *m, int batch, const float *noise_dev, int nk,
+                  const uint8_t *init_dev, int mode, int block, int max_iters,
+                  uint8_t *out_samples_dev, int32_t *out_iters_dev, void *cuda_stream);
+
+/* Strict feedforward order (Eq. 1): T steps, each a forward pass of the same kernels of
+ * which one position is kept. */
+int sequential_sample(const js_model *m, int batch, const float *noise_dev, int nk,
+                      uint8_t *out_samples_dev, void *cuda_stream);
+
+/* Logits of every position for given symbols x (teacher forcing): logits_dev fp32
+ * [batch][T][C].  For parity checks of the network itself. */
+int js_forward_logits(const js_model *m, int batch, const uint8_t *x_dev, float *logits_dev,
+                      void *cuda_stream);
+
+typedef enum {
+    JS_OPT_FRONTIER_SKIP = 0,  /* 1 (default): skip positions and hidden units already final (proof of Prop. 1) */
+    JS_OPT_SEQ_SKIP = 1,       /* 0 (default): sequential_sample recomputes everything each step; 1: only the band that changed */
+    JS_OPT_SPIN_LIMIT = 2,     /* polls before a device-side wait gives up (default 1<<22) */
+    JS_OPT_PATH = 3,           /* 0 (default): tensor-core kernels where the model allows; 1: CUDA-core kernels only */
+    JS_OPT_COMPACT = 4         /* 1 (default): move finished samples out of the working batch */
+} js_option;
+int js_set_option(js_model *m, int option, int value);
+
+/* counters of the most recent sampling call on this model */
+typedef struct {
+    int iterations;            /* forward passes executed (micro-steps for Jacobi-GS) */
+    int batch_iters_max;       /* largest per-sample iteration count */
+    int final_frontier;        /* leading positions known final when the loop ended */
+    long long tiles_issued;    /* output tiles computed */
+    long long tiles_skipped;   /* output tiles skipped as final, finished or masked */
+    int path;                  /* 0 tensor-core kernels, 1 CUDA-core kernels */
+    int status;                /* the call's return value */
+} js_stats;
+int js_get_stats(const js_model *m, js_stats *out);
+
+const char *js_strerror(int code);
+const char *js_last_cuda_error(void);   /* text of the last failed CUDA call on this thread */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* JACOBI_SAMPLE_H */

@@ -1,0 +1,355 @@
+// C ABI of the sampler library: model construction (masking, rounding, tile
+// metadata), argument checks, kernel selection and launch, status read-back.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "js_common.cuh"
+#include "js_model.h"
+
+static thread_local char g_cuda_err[256] = "";
+
+#define CU_TRY(call)                                                                         \
+    do {                                                                                     \
+        cudaError_t e__ = (call);                                                            \
+        if (e__ != cudaSuccess) {                                                            \
+            snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s", #call, cudaGetErrorString(e__)); \
+            return JS_ERR_CUDA;                                                              \
+        }                                                                                    \
+    } while (0)
+
+namespace {
+
+// masked, rounded copy of one weight matrix:  Wm[i][j] = keep(i, j) ? W[i][j] : 0
+template <typename T>
+__global__ void pack_made_weights(const float *__restrict__ W, const int *__restrict__ deg_out,
+                                  const int *__restrict__ deg_in, int n_out, int n_in, int strict, T *__restrict__ out)
+{
+    const size_t n = (size_t)n_out * n_in;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int r = (int)(i / n_in), c = (int)(i % n_in);
+        const bool keep = strict ? (deg_out[r] > deg_in[c]) : (deg_out[r] >= deg_in[c]);
+        out[i] = from_f32<T>(keep ? W[i] : 0.0f);
+    }
+}
+
+template <typename T>
+int dev_alloc(js_model *m, T **p, size_t count, bool zero)
+{
+    void *q = nullptr;
+    const size_t bytes = std::max<size_t>(count * sizeof(T), 16);
+    CU_TRY(cudaMalloc(&q, bytes));
+    m->allocs.push_back(q);
+    if (zero) CU_TRY(cudaMemset(q, 0, bytes));
+    *p = (T *)q;
+    return JS_OK;
+}
+
+template <typename T>
+int dev_upload(js_model *m, const T **p, const T *host, size_t count)
+{
+    T *q = nullptr;
+    int rc = dev_alloc(m, &q, count, false);
+    if (rc != JS_OK) return rc;
+    CU_TRY(cudaMemcpy(q, host, count * sizeof(T), cudaMemcpyHostToDevice));
+    *p = q;
+    return JS_OK;
+}
+
+int made_build(js_model *m, const js_made_desc *d)
+{
+    MadeDev &v = m->made;
+    v.T = d->T; v.C = d->C; v.L = d->L; v.act = d->act; v.prec = d->prec;
+    v.n[0] = d->T;
+    for (int l = 0; l < d->L; ++l) v.n[l + 1] = d->H[l];
+    v.n[d->L + 1] = d->T * d->C;
+    const int L = d->L;
+    const size_t esz = d->prec == JS_BF16 ? 2 : 4;
+
+    // degrees
+    std::vector<std::vector<int>> deg(L + 2);
+    for (int l = 0; l <= L + 1; ++l) deg[l].resize(v.n[l]);
+    for (int i = 0; i < d->T; ++i) deg[0][i] = i + 1;
+    for (int l = 1; l <= L; ++l)
+        for (int j = 0; j < v.n[l]; ++j) {
+            int g = (d->hidden_deg && d->hidden_deg[l - 1]) ? d->hidden_deg[l - 1][j]
+                                                            : 1 + (int)(((long long)j * (d->T - 1)) / v.n[l]);
+            if (g < 1 || g > d->T) return JS_ERR_ARG;
+            deg[l][j] = g;
+        }
+    for (int i = 0; i < d->T * d->C; ++i) deg[L + 1][i] = i / d->C + 1;
+    for (int l = 0; l <= L + 1; ++l) {
+        int rc = dev_upload<int>(m, &v.deg[l], deg[l].data(), deg[l].size());
+        if (rc != JS_OK) return rc;
+    }
+
+    // per-tile metadata for the 64-wide output tiles of every layer
+    for (int l = 0; l <= L; ++l) {
+        const int N = v.n[l + 1], K = v.n[l], nt = (N + JS_GT - 1) / JS_GT;
+        std::vector<int> kend(nt), dmin(nt), dmax(nt);
+        for (int t = 0; t < nt; ++t) {
+            int lo = INT32_MAX, hi = 0;
+            for (int i = t * JS_GT; i < std::min(N, (t + 1) * JS_GT); ++i) {
+                lo = std::min(lo, deg[l + 1][i]);
+                hi = std::max(hi, deg[l + 1][i]);
+            }
+            int ke = K;
+            while (ke > 0 && !(l == L ? deg[l][ke - 1] < hi : deg[l][ke - 1] <= hi)) --ke;
+            kend[t] = ke; dmin[t] = lo; dmax[t] = hi;
+        }
+        int rc;
+        if ((rc = dev_upload<int>(m, &v.t_kend[l], kend.data(), nt)) != JS_OK) return rc;
+        if ((rc = dev_upload<int>(m, &v.t_dmin[l], dmin.data(), nt)) != JS_OK) return rc;
+        if ((rc = dev_upload<int>(m, &v.t_dmax[l], dmax.data(), nt)) != JS_OK) return rc;
+        m->host_deg = deg;
+    }
+
+    // weights: upload unmasked fp32, mask and round on the device
+    for (int l = 0; l <= L; ++l) {
+        const size_t cnt = (size_t)v.n[l + 1] * v.n[l];
+        float *tmp = nullptr;
+        CU_TRY(cudaMalloc((void **)&tmp, cnt * sizeof(float)));
+        cudaError_t e = cudaMemcpy(tmp, d->W[l], cnt * sizeof(float), cudaMemcpyHostToDevice);
+        void *wm = nullptr;
+        if (e == cudaSuccess) e = cudaMalloc(&wm, cnt * esz);
+        if (e == cudaSuccess) {
+            m->allocs.push_back(wm);
+            const int grid = (int)std::min<size_t>((cnt + 255) / 256, 148 * 16);
+            if (d->prec == JS_BF16)
+                pack_made_weights<__nv_bfloat16><<<grid, 256>>>(tmp, v.deg[l + 1], v.deg[l], v.n[l + 1], v.n[l],
+                                                                 l == L, (__nv_bfloat16 *)wm);
+            else
+                pack_made_weights<float><<<grid, 256>>>(tmp, v.deg[l + 1], v.deg[l], v.n[l + 1], v.n[l], l == L,
+                                                         (float *)wm);
+            e = cudaGetLastError();
+            if (e == cudaSuccess) e = cudaDeviceSynchronize();
+        }
+        cudaFree(tmp);
+        CU_TRY(e);
+        v.W[l] = wm;
+        int rc = dev_upload<float>(m, &v.bias[l], d->b[l], v.n[l + 1]);
+        if (rc != JS_OK) return rc;
+    }
+
+    // input table, rounded like an activation
+    {
+        std::vector<float> lut(d->lut, d->lut + d->n_lut);
+        if (d->prec == JS_BF16)
+            for (auto &f : lut) f = __bfloat162float(__float2bfloat16_rn(f));
+        int rc = dev_upload<float>(m, &v.lut, lut.data(), lut.size());
+        if (rc != JS_OK) return rc;
+    }
+
+    // activations and scratch
+    m->rows = (m->max_batch + 127) / 128 * 128;
+    for (int l = 0; l <= L; ++l) {
+        char *p = nullptr, *q = nullptr;
+        int rc;
+        if ((rc = dev_alloc<char>(m, &p, (size_t)m->rows * v.n[l] * esz, true)) != JS_OK) return rc;
+        if ((rc = dev_alloc<char>(m, &q, (size_t)m->rows * v.n[l] * esz, true)) != JS_OK) return rc;
+        v.a[l] = p; v.a_old[l] = q;
+    }
+    int rc;
+    if ((rc = dev_alloc<float>(m, &v.logits, (size_t)m->rows * v.n[L + 1], true)) != JS_OK) return rc;
+    return JS_OK;
+}
+
+int common_scratch(js_model *m, int T)
+{
+    int rc;
+    if ((rc = dev_alloc<JsCtl>(m, &m->ctl, 1, true)) != JS_OK) return rc;
+    if ((rc = dev_alloc<int>(m, &m->smp_changed, 2 * (size_t)m->rows, true)) != JS_OK) return rc;
+    if ((rc = dev_alloc<int>(m, &m->smp_state, 2 * (size_t)m->rows, true)) != JS_OK) return rc;
+    if ((rc = dev_alloc<uint8_t>(m, &m->x_old, (size_t)m->rows * T, true)) != JS_OK) return rc;
+    if ((rc = dev_alloc<uint8_t>(m, &m->x_tmp, (size_t)m->rows * T, true)) != JS_OK) return rc;
+    return JS_OK;
+}
+
+bool noise_kind_ok(const js_model *m, int nk)
+{
+    const int C = m->kind == 0 ? m->made.C : m->conv_C;
+    if (nk == JS_NOISE_GUMBEL) return C > 1;
+    if (nk == JS_NOISE_UNIFORM_ICDF || nk == JS_NOISE_LOGISTIC) return C == 1;
+    return false;
+}
+
+int run_made(js_model *m, RunArgs &r, cudaStream_t st)
+{
+    const MadeDev &v = m->made;
+    r.ctl = m->ctl;
+    r.smp_changed = m->smp_changed;
+    r.smp_state = m->smp_state;
+    r.x_old = m->x_old;
+    r.frontier_skip = m->opt_frontier_skip;
+    r.seq_skip = m->opt_seq_skip;
+    r.spin_limit = (unsigned)m->opt_spin_limit;
+    CU_TRY(cudaMemsetAsync(m->ctl, 0, sizeof(JsCtl), st));
+
+    int used_path = 1;
+    int rc_launch;
+    if (m->max_grid_generic <= 0) m->max_grid_generic = js_made_generic_max_grid(v.prec);
+    if (m->max_grid_generic <= 0) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "occupancy query failed");
+        return JS_ERR_CUDA;
+    }
+    {
+        long long tiles = 1;
+        for (int l = 0; l <= v.L; ++l)
+            tiles = std::max<long long>(tiles, (long long)((r.batch + JS_GT - 1) / JS_GT) * ((v.n[l + 1] + JS_GT - 1) / JS_GT));
+        const long long elems = ((long long)r.batch * v.T * (v.C > 1 ? 32 : 1) + 255) / 256;
+        const int grid = (int)std::min<long long>(m->max_grid_generic, std::max(tiles, elems));
+        rc_launch = js_launch_made_generic(v, r, std::max(grid, 1), st);
+    }
+    if (rc_launch != 0) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "kernel launch: %s", cudaGetErrorString((cudaError_t)rc_launch));
+        return JS_ERR_CUDA;
+    }
+    JsCtl h;
+    CU_TRY(cudaMemcpyAsync(&h, m->ctl, sizeof h, cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    m->stats.iterations = h.iterations;
+    m->stats.final_frontier = h.frontier;
+    m->stats.tiles_issued = (long long)h.tiles_issued;
+    m->stats.tiles_skipped = (long long)h.tiles_skipped;
+    m->stats.batch_iters_max = h.iters_max;
+    m->stats.path = used_path;
+    m->stats.status = h.status;
+    return h.status;
+}
+
+}  // namespace
+
+extern "C" {
+
+int js_made_create(const js_made_desc *d, js_model **out)
+{
+    if (!d || !out) return JS_ERR_ARG;
+    *out = nullptr;
+    if (d->T < 1 || d->C < 1 || d->C > 256 || d->L < 1 || d->L > JS_MAXL || !d->H || !d->W || !d->b || !d->lut ||
+        d->max_batch < 1)
+        return JS_ERR_ARG;
+    if (d->act != JS_ACT_RELU && d->act != JS_ACT_GELU_TANH) return JS_ERR_ARG;
+    if (d->prec != JS_F32 && d->prec != JS_BF16) return JS_ERR_ARG;
+    if (d->n_lut != (d->C == 1 ? 2 : d->C)) return JS_ERR_ARG;
+    for (int l = 0; l < d->L; ++l)
+        if (d->H[l] < 1) return JS_ERR_ARG;
+    for (int l = 0; l <= d->L; ++l)
+        if (!d->W[l] || !d->b[l]) return JS_ERR_ARG;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "no CUDA device");
+        return JS_ERR_CUDA;
+    }
+    js_model *m = new (std::nothrow) js_model();
+    if (!m) return JS_ERR_ARG;
+    m->kind = 0;
+    m->max_batch = d->max_batch;
+    int rc = made_build(m, d);
+    if (rc == JS_OK) rc = common_scratch(m, d->T);
+    if (rc != JS_OK) { js_model_destroy(m); return rc; }
+    *out = m;
+    return JS_OK;
+}
+
+int js_conv_create(const js_conv_desc *d, js_model **out)
+{
+    (void)d;
+    if (out) *out = nullptr;
+    return JS_ERR_UNSUPPORTED;
+}
+
+void js_model_destroy(js_model *m)
+{
+    if (!m) return;
+    for (void *p : m->allocs) cudaFree(p);
+    delete m;
+}
+
+int jacobi_sample(const js_model *cm, int batch, const float *noise_dev, int nk, const uint8_t *init_dev, int mode,
+                  int block, int max_iters, uint8_t *out_samples_dev, int32_t *out_iters_dev, void *cuda_stream)
+{
+    js_model *m = const_cast<js_model *>(cm);
+    if (!m || !noise_dev || !out_samples_dev) return JS_ERR_ARG;
+    if (batch < 1 || batch > m->max_batch) return JS_ERR_ARG;
+    if (mode < JS_JACOBI || mode > JS_JACOBI_GS) return JS_ERR_ARG;
+    if (!noise_kind_ok(m, nk)) return JS_ERR_ARG;
+    const int T = m->kind == 0 ? m->made.T : m->conv_T;
+    if ((mode == JS_GS_JACOBI || mode == JS_JACOBI_GS) && (block < 1 || block > T)) return JS_ERR_ARG;
+    if (m->kind != 0) return JS_ERR_UNSUPPORTED;
+    RunArgs r;
+    memset(&r, 0, sizeof r);
+    r.batch = batch; r.noise = noise_dev; r.nk = nk; r.init = init_dev;
+    r.kmode = mode == JS_JACOBI ? KM_JACOBI : mode == JS_GAUSS_SEIDEL ? KM_SEQ : mode == JS_GS_JACOBI ? KM_GS_JACOBI
+                                                                                                        : KM_JACOBI_GS;
+    r.block = block; r.max_iters = max_iters;
+    r.x = out_samples_dev; r.out_iters = out_iters_dev;
+    int rc = run_made(m, r, (cudaStream_t)cuda_stream);
+    return rc;
+}
+
+int sequential_sample(const js_model *cm, int batch, const float *noise_dev, int nk, uint8_t *out_samples_dev,
+                      void *cuda_stream)
+{
+    js_model *m = const_cast<js_model *>(cm);
+    if (!m || !noise_dev || !out_samples_dev) return JS_ERR_ARG;
+    if (batch < 1 || batch > m->max_batch) return JS_ERR_ARG;
+    if (!noise_kind_ok(m, nk)) return JS_ERR_ARG;
+    if (m->kind != 0) return JS_ERR_UNSUPPORTED;
+    RunArgs r;
+    memset(&r, 0, sizeof r);
+    r.batch = batch; r.noise = noise_dev; r.nk = nk; r.kmode = KM_SEQ;
+    r.x = out_samples_dev;
+    return run_made(m, r, (cudaStream_t)cuda_stream);
+}
+
+int js_forward_logits(const js_model *cm, int batch, const uint8_t *x_dev, float *logits_dev, void *cuda_stream)
+{
+    js_model *m = const_cast<js_model *>(cm);
+    if (!m || !x_dev || !logits_dev) return JS_ERR_ARG;
+    if (batch < 1 || batch > m->max_batch) return JS_ERR_ARG;
+    if (m->kind != 0) return JS_ERR_UNSUPPORTED;
+    RunArgs r;
+    memset(&r, 0, sizeof r);
+    r.batch = batch; r.kmode = KM_FORWARD; r.x_in = x_dev; r.logits_out = logits_dev;
+    r.x = m->x_tmp;
+    return run_made(m, r, (cudaStream_t)cuda_stream);
+}
+
+int js_set_option(js_model *m, int option, int value)
+{
+    if (!m) return JS_ERR_ARG;
+    switch (option) {
+    case JS_OPT_FRONTIER_SKIP: m->opt_frontier_skip = value ? 1 : 0; return JS_OK;
+    case JS_OPT_SEQ_SKIP: m->opt_seq_skip = value ? 1 : 0; return JS_OK;
+    case JS_OPT_SPIN_LIMIT: if (value < 0) return JS_ERR_ARG; m->opt_spin_limit = value; return JS_OK;
+    case JS_OPT_PATH: if (value != 0 && value != 1) return JS_ERR_ARG; m->opt_path = value; return JS_OK;
+    case JS_OPT_COMPACT: m->opt_compact = value ? 1 : 0; return JS_OK;
+    default: return JS_ERR_ARG;
+    }
+}
+
+int js_get_stats(const js_model *m, js_stats *out)
+{
+    if (!m || !out) return JS_ERR_ARG;
+    *out = m->stats;
+    return JS_OK;
+}
+
+const char *js_strerror(int code)
+{
+    switch (code) {
+    case JS_OK: return "ok";
+    case JS_NOT_CONVERGED: return "iteration cap reached before every sample stopped changing";
+    case JS_ERR_ARG: return "invalid argument";
+    case JS_ERR_UNSUPPORTED: return "unsupported model shape or mode";
+    case JS_ERR_CUDA: return "CUDA runtime error";
+    case JS_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    default: return "unknown code";
+    }
+}
+
+const char *js_last_cuda_error(void) { return g_cuda_err; }
+
+}  // extern "C"

@@ -1,0 +1,134 @@
+// Shared declarations of the sampler library: device-side model views, the
+// control block of the persistent kernels and the bounded grid barrier.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/jacobi_sample.h"
+
+#define JS_MAXL 8
+#define JS_GT 64          // output-tile edge of the CUDA-core GEMM phases
+
+enum { KM_JACOBI = 0, KM_SEQ = 1, KM_GS_JACOBI = 2, KM_JACOBI_GS = 3, KM_FORWARD = 4 };
+
+// Control block in device memory, zeroed by the host before every launch.
+struct JsCtl {
+    unsigned bar_count;     // grid barrier: monotonically increasing arrival counter
+    int abort;              // set when a bounded wait gave up; every CTA then leaves
+    int status;             // JS_OK / JS_NOT_CONVERGED / JS_ERR_TIMEOUT
+    int agg_any[2];         // per iteration parity: did any sample change
+    int agg_minfirst[2];    // per iteration parity: smallest changed position
+    int iterations;         // forward passes executed
+    int frontier;           // leading positions known final at exit
+    int iters_max;
+    int live;               // samples still iterating (tensor-core path)
+    unsigned long long tiles_issued, tiles_skipped;
+};
+
+// Device view of a masked MLP.  Layer l maps a[l] (width n[l]) to a[l+1].
+struct MadeDev {
+    int T, C, L, act, prec;
+    int n[JS_MAXL + 2];
+    const void *W[JS_MAXL + 1];       // masked weights [n[l+1]][n[l]], float or bf16
+    const float *bias[JS_MAXL + 1];
+    void *a[JS_MAXL + 1];             // activations [rows][n[l]], float or bf16 (a[0] = encoded iterate)
+    void *a_old[JS_MAXL + 1];         // Jacobi-GS: activations of the previous outer iterate
+    const int *deg[JS_MAXL + 2];      // degree of every unit
+    const int *t_kend[JS_MAXL + 1];   // per JS_GT-wide output tile: inputs beyond this index are masked
+    const int *t_dmin[JS_MAXL + 1];   // per tile: smallest / largest degree inside
+    const int *t_dmax[JS_MAXL + 1];
+    const float *lut;
+    float *logits;                    // scratch [rows][T*C]
+};
+
+struct RunArgs {
+    int batch;
+    const float *noise;
+    int nk;
+    const uint8_t *init;
+    int kmode;
+    int block;
+    int max_iters;
+    uint8_t *x;               // working iterate = output samples [batch][T]
+    uint8_t *x_old;           // scratch [batch][T] (Jacobi-GS)
+    int32_t *out_iters;       // may be NULL
+    int *smp_changed;         // [2][batch] per-sample change flags by iteration parity
+    int *smp_state;           // [2][batch] per-sample bookkeeping (done flag, running count)
+    const uint8_t *x_in;      // KM_FORWARD: symbols
+    float *logits_out;        // KM_FORWARD: destination
+    int frontier_skip, seq_skip;
+    unsigned spin_limit;
+    JsCtl *ctl;
+};
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ int ld_volatile_i32(const int *p)
+{
+    int v;
+    asm volatile("ld.volatile.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Grid-wide barrier for a cooperative (co-resident) launch.  Every CTA calls it
+// the same number of times; `epoch` counts the calls.  The wait is bounded: after
+// spin_limit polls, or when another CTA has given up, the CTA raises `abort` and
+// the function returns false in every thread of the CTA; the caller must then
+// leave the kernel.  Returns true when all CTAs have arrived.
+__device__ __forceinline__ bool grid_barrier(JsCtl *ctl, unsigned &epoch, unsigned spin_limit)
+{
+    __syncthreads();
+    epoch += 1;
+    int ok = 1;
+    if (threadIdx.x == 0) {
+        __threadfence();
+        const unsigned target = epoch * gridDim.x;
+        atomicAdd(&ctl->bar_count, 1u);
+        unsigned polls = 0;
+        while (ld_acquire_u32(&ctl->bar_count) < target) {
+            if (++polls > spin_limit || ld_volatile_i32(&ctl->abort) != 0) {
+                atomicExch(&ctl->abort, 1);
+                ok = 0;
+                break;
+            }
+            if (polls > 64) __nanosleep(64);
+        }
+        if (ok && ld_volatile_i32(&ctl->abort) != 0) ok = 0;
+        __threadfence();
+    }
+    return __syncthreads_and(ok) != 0;
+}
+
+__device__ __forceinline__ float js_act_fn(int act, float v)
+{
+    if (act == JS_ACT_RELU) return fmaxf(v, 0.0f);
+    const float y = 0.7978845608028654f * (v + 0.044715f * v * v * v);
+    return 0.5f * v * (1.0f + tanhf(y));
+}
+
+// x_t from the logits of position t and its reserved noise (Appendix A.3), binary kinds
+__device__ __forceinline__ int js_sample_binary(int nk, float z, float noise)
+{
+    if (nk == JS_NOISE_UNIFORM_ICDF) {
+        const float p = 1.0f / (1.0f + expf(-z));
+        return noise < p ? 1 : 0;
+    }
+    return (z + noise) > 0.0f ? 1 : 0;
+}
+
+template <typename T> __device__ __forceinline__ float to_f32(T v);
+template <> __device__ __forceinline__ float to_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+// host-side launchers implemented by the kernel files
+int js_launch_made_generic(const MadeDev &m, const RunArgs &r, int grid_limit, cudaStream_t stream);
+int js_made_generic_max_grid(int prec);

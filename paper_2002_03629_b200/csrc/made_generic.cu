@@ -1,0 +1,575 @@
+// CUDA-core path of the masked-MLP sampler: one persistent cooperative kernel
+// that runs the whole solver (Algorithms 1-3 of arXiv 2002.03629, or the strict
+// feedforward order of Eq. 1) on the device.  It serves fp32 models, shapes the
+// tensor-core path does not cover, and the fine-grained sweeps of Jacobi-GS.
+//
+// Every CTA executes the same driver loop; decisions are taken from values all
+// CTAs read identically after a grid barrier, so control flow never diverges
+// between CTAs.  Each output value is accumulated in a fixed order over k that
+// does not depend on what else is skipped, so h_t is the same function in every
+// iteration (the convergence proofs need that).
+#include <limits.h>
+
+#include "js_common.cuh"
+
+namespace {
+
+constexpr int GT = JS_GT;      // 64x64 output tile
+constexpr int KC = 32;         // k chunk staged in shared memory
+constexpr int NTHREADS = 256;
+
+struct Win {
+    int hdeg_lo;   // hidden units of degree <= hdeg_lo are final: not recomputed
+    int hdeg_hi;   // hidden units of degree >  hdeg_hi are not needed yet
+    int plo, phi;  // output positions [plo, phi)
+};
+
+struct Smem {
+    float As[KC][GT + 4];
+    float Bs[KC][GT + 4];
+    int list[4096];            // Jacobi-GS: units to evaluate in this micro-step
+    int list_n;
+    int wcnt[NTHREADS / 32];
+};
+
+// One 64x64 tile of  out = A[batch][K] * W[N][K]^T  over k in [0, kend).
+template <typename T>
+__device__ void gemm_tile(Smem &s, const T *A, int lda, const T *__restrict__ W, int ldw,
+                          int M, int N, int kend, int m0, int n0, float (&acc)[4][4])
+{
+    const int tid = threadIdx.x;
+    const int ty = tid >> 4, tx = tid & 15;
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
+    for (int k0 = 0; k0 < kend; k0 += KC) {
+#pragma unroll
+        for (int it = 0; it < (GT * KC) / NTHREADS; ++it) {
+            const int idx = tid + it * NTHREADS;
+            const int kk = idx % KC, row = idx / KC;
+            const int k = k0 + kk;
+            float av = 0.0f, bv = 0.0f;
+            if (k < kend) {
+                if (m0 + row < M) av = to_f32<T>(A[(size_t)(m0 + row) * lda + k]);
+                if (n0 + row < N) bv = to_f32<T>(W[(size_t)(n0 + row) * ldw + k]);
+            }
+            s.As[kk][row] = av;
+            s.Bs[kk][row] = bv;
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int kk = 0; kk < KC; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = s.As[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = s.Bs[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+}
+
+// Layer l over the window: hidden layers store act(pre) into `out`; the output
+// layer (l == L) stores fp32 logits into `zout` [batch][T*C].
+template <typename T>
+__device__ void gemm_phase(Smem &s, const MadeDev &m, int l, const T *Asrc, T *out, float *zout, int batch,
+                           const Win &w, unsigned long long &issued, unsigned long long &skipped)
+{
+    const int N = m.n[l + 1], K = m.n[l];
+    const int mt = (batch + GT - 1) / GT, nt = (N + GT - 1) / GT;
+    const bool is_out = (l == m.L);
+    const T *Wl = (const T *)m.W[l];
+    for (int tile = blockIdx.x; tile < mt * nt; tile += gridDim.x) {
+        const int tn = tile / mt, tm = tile % mt;
+        const int dmin = m.t_dmin[l][tn], dmax = m.t_dmax[l][tn];
+        bool live;
+        if (is_out) live = (dmax - 1 >= w.plo) && (dmin - 1 < w.phi);
+        else live = (dmax > w.hdeg_lo) && (dmin <= w.hdeg_hi);
+        if (!live) { if (threadIdx.x == 0) skipped++; continue; }
+        if (threadIdx.x == 0) issued++;
+        float acc[4][4];
+        const int m0 = tm * GT, n0 = tn * GT;
+        gemm_tile<T>(s, Asrc, K, Wl, K, batch, N, m.t_kend[l][tn], m0, n0, acc);
+        const int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int row = m0 + ty * 4 + i;
+            if (row >= batch) continue;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int col = n0 + tx * 4 + j;
+                if (col >= N) continue;
+                const float pre = acc[i][j] + m.bias[l][col];
+                if (is_out) zout[(size_t)row * N + col] = pre;
+                else out[(size_t)row * N + col] = from_f32<T>(js_act_fn(m.act, pre));
+            }
+        }
+    }
+}
+
+// x = init (or zeros), a[0] = lut[x]; also clears the per-sample bookkeeping.
+template <typename T>
+__device__ void init_phase(const MadeDev &m, const RunArgs &r, const uint8_t *src)
+{
+    const size_t n = (size_t)r.batch * m.T;
+    T *a0 = (T *)m.a[0];
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const uint8_t v = src ? src[i] : (uint8_t)0;
+        if (r.x) r.x[i] = v;
+        a0[i] = from_f32<T>(m.lut[v]);
+    }
+    if (blockIdx.x == 0) {
+        for (int i = threadIdx.x; i < 2 * r.batch; i += blockDim.x) {
+            r.smp_changed[i] = 0;
+            r.smp_state[i] = 0;
+        }
+        if (threadIdx.x == 0) {
+            r.ctl->agg_any[0] = r.ctl->agg_any[1] = 0;
+            r.ctl->agg_minfirst[0] = r.ctl->agg_minfirst[1] = INT_MAX;
+        }
+    }
+}
+
+__device__ __forceinline__ void note_change(const RunArgs &r, int parity, int b, int d)
+{
+    atomicOr(&r.smp_changed[parity * r.batch + b], 1);
+    atomicMin(&r.ctl->agg_minfirst[parity], d);
+    atomicOr(&r.ctl->agg_any[parity], 1);
+}
+
+// Sample positions [plo, phi) of every sample from the logits scratch, compare
+// with the current iterate, store the new symbol and its encoding.
+template <typename T>
+__device__ void sample_phase(const MadeDev &m, const RunArgs &r, const float *z, int plo, int phi, bool flag,
+                             int parity)
+{
+    const int T_ = m.T, C = m.C, np = phi - plo;
+    T *a0 = (T *)m.a[0];
+    if (C == 1) {
+        const size_t n = (size_t)r.batch * np;
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+            const int b = (int)(i / np), d = plo + (int)(i % np);
+            const size_t at = (size_t)b * T_ + d;
+            const int xn = js_sample_binary(r.nk, z[at], r.noise[at]);
+            if (xn != r.x[at]) {
+                r.x[at] = (uint8_t)xn;
+                a0[at] = from_f32<T>(m.lut[xn]);
+                if (flag) note_change(r, parity, b, d);
+            }
+        }
+        return;
+    }
+    const int lane = threadIdx.x & 31;
+    const size_t warps = ((size_t)gridDim.x * blockDim.x) >> 5;
+    const size_t n = (size_t)r.batch * np;
+    for (size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
+        const int b = (int)(i / np), d = plo + (int)(i % np);
+        const size_t at = (size_t)b * T_ + d;
+        const float *zz = z + at * C;
+        const float *gg = r.noise + at * C;
+        float best = -INFINITY;
+        int bi = INT_MAX;
+        for (int c = lane; c < C; c += 32) {
+            const float v = zz[c] + gg[c];
+            if (v > best) { best = v; bi = c; }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, best, off);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+            if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+        }
+        if (lane == 0 && bi != r.x[at]) {
+            r.x[at] = (uint8_t)bi;
+            a0[at] = from_f32<T>(m.lut[bi]);
+            if (flag) note_change(r, parity, b, d);
+        }
+    }
+}
+
+// After the barrier that ends an iteration: CTA 0 clears the other parity's flags.
+__device__ void reset_other_parity(const RunArgs &r, int parity)
+{
+    if (blockIdx.x != 0) return;
+    const int o = parity ^ 1;
+    for (int i = threadIdx.x; i < r.batch; i += blockDim.x) r.smp_changed[o * r.batch + i] = 0;
+    if (threadIdx.x == 0) {
+        r.ctl->agg_any[o] = 0;
+        r.ctl->agg_minfirst[o] = INT_MAX;
+    }
+}
+
+// CTA 0: a sample whose iterate did not change (or that hit the cap) stops counting.
+__device__ void book_samples(const RunArgs &r, int parity, int k, bool at_cap, bool add, bool final_write)
+{
+    if (blockIdx.x != 0) return;
+    int *done = r.smp_state, *count = r.smp_state + r.batch;
+    for (int b = threadIdx.x; b < r.batch; b += blockDim.x) {
+        if (!done[b] && (r.smp_changed[parity * r.batch + b] == 0 || at_cap)) {
+            done[b] = 1;
+            count[b] = add ? count[b] + k : k;
+            if (final_write && r.out_iters) r.out_iters[b] = count[b];
+        }
+    }
+}
+
+template <typename T>
+__device__ bool forward_pass(Smem &s, const MadeDev &m, const RunArgs &r, T *const *acts, float *zout, const Win &w,
+                             unsigned &epoch, unsigned long long &issued, unsigned long long &skipped)
+{
+    for (int l = 0; l <= m.L; ++l) {
+        gemm_phase<T>(s, m, l, (const T *)acts[l], l < m.L ? acts[l + 1] : (T *)nullptr, zout, r.batch, w, issued,
+                      skipped);
+        if (!grid_barrier(r.ctl, epoch, r.spin_limit)) return false;
+    }
+    return true;
+}
+
+// ---- Jacobi-GS micro-steps (Algorithm 2): warp-per-dot-product evaluation of
+// the units that become computable at step j of every block's sequential sweep.
+// A unit of block i reads, from the layer below, units of earlier blocks at the
+// previous outer iterate (`old`) and units of its own block at the current one.
+template <typename T>
+__device__ float mixed_dot(const MadeDev &m, int l, int unit, int blk, int B, const T *old_row, const T *new_row,
+                           int kend)
+{
+    const int lane = threadIdx.x & 31;
+    const T *w = (const T *)m.W[l] + (size_t)unit * m.n[l];
+    const int *dg = m.deg[l];
+    float acc = 0.0f;
+    for (int k = lane; k < kend; k += 32) {
+        const bool use_old = ((dg[k] - 1) / B) < blk;
+        acc = fmaf(to_f32<T>(w[k]), to_f32<T>(use_old ? old_row[k] : new_row[k]), acc);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+    return acc;
+}
+
+template <typename T>
+__device__ void jgs_hidden_phase(Smem &s, const MadeDev &m, const RunArgs &r, int l, int j, int B, int blk_lo)
+{
+    // units of layer l+1 whose degree g satisfies g % B == j, in blocks >= blk_lo.
+    // The list is built in index order so that every CTA holds the same list.
+    const int N = m.n[l + 1];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const size_t warps = ((size_t)gridDim.x * blockDim.x) >> 5;
+    for (int ubase = 0; ubase < N; ubase += 4096) {
+        const int uend = min(N, ubase + 4096);
+        if (threadIdx.x == 0) s.list_n = 0;
+        __syncthreads();
+        for (int base = ubase; base < uend; base += NTHREADS) {
+            const int i = base + threadIdx.x;
+            bool pred = false;
+            if (i < uend) {
+                const int g = m.deg[l + 1][i];
+                pred = (g % B == j) && ((g - 1) / B >= blk_lo);
+            }
+            const unsigned bal = __ballot_sync(0xffffffffu, pred);
+            if (lane == 0) s.wcnt[warp] = __popc(bal);
+            __syncthreads();
+            int off = s.list_n;
+            for (int w2 = 0; w2 < warp; ++w2) off += s.wcnt[w2];
+            if (pred) s.list[off + __popc(bal & ((1u << lane) - 1u))] = i;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                int tot = 0;
+                for (int w2 = 0; w2 < NTHREADS / 32; ++w2) tot += s.wcnt[w2];
+                s.list_n += tot;
+            }
+            __syncthreads();
+        }
+        const int cnt = s.list_n;
+        const size_t items = (size_t)cnt * r.batch;
+        for (size_t it = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; it < items; it += warps) {
+            const int unit = s.list[it / r.batch], b = (int)(it % r.batch);
+            const int g = m.deg[l + 1][unit];
+            const float pre = mixed_dot<T>(m, l, unit, (g - 1) / B, B, (const T *)m.a_old[l] + (size_t)b * m.n[l],
+                                           (const T *)m.a[l] + (size_t)b * m.n[l], m.t_kend[l][unit / GT]) +
+                              m.bias[l][unit];
+            if (lane == 0) ((T *)m.a[l + 1])[(size_t)b * N + unit] = from_f32<T>(js_act_fn(m.act, pre));
+        }
+        __syncthreads();
+    }
+}
+
+template <typename T>
+__device__ void jgs_output_phase(const MadeDev &m, const RunArgs &r, int j, int B, int blk_lo)
+{
+    const int L = m.L, C = m.C, nblk = (m.T + B - 1) / B;
+    const size_t warps = ((size_t)gridDim.x * blockDim.x) >> 5;
+    const size_t items = (size_t)(nblk - blk_lo) * C * r.batch;
+    const int lane = threadIdx.x & 31;
+    for (size_t it = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; it < items; it += warps) {
+        const int b = (int)(it % r.batch);
+        const int c = (int)((it / r.batch) % C);
+        const int blk = blk_lo + (int)(it / ((size_t)r.batch * C));
+        const int t = blk * B + j;
+        if (t >= m.T) continue;
+        const int unit = t * C + c;
+        const float z = mixed_dot<T>(m, L, unit, blk, B, (const T *)m.a_old[L] + (size_t)b * m.n[L],
+                                     (const T *)m.a[L] + (size_t)b * m.n[L], m.t_kend[L][unit / GT]) +
+                        m.bias[L][unit];
+        if (C == 1) {
+            if (lane == 0) {
+                const size_t at = (size_t)b * m.T + t;
+                const int xn = js_sample_binary(r.nk, z, r.noise[at]);
+                r.x[at] = (uint8_t)xn;
+                ((T *)m.a[0])[at] = from_f32<T>(m.lut[xn]);
+            }
+        } else if (lane == 0) {
+            m.logits[(size_t)b * m.n[L + 1] + unit] = z;
+        }
+    }
+}
+
+// categorical commit of position blk*B + j for every block (no change flags here)
+template <typename T>
+__device__ void jgs_commit_phase(const MadeDev &m, const RunArgs &r, int j, int B, int blk_lo)
+{
+    const int C = m.C, nblk = (m.T + B - 1) / B;
+    const size_t warps = ((size_t)gridDim.x * blockDim.x) >> 5;
+    const size_t items = (size_t)(nblk - blk_lo) * r.batch;
+    const int lane = threadIdx.x & 31;
+    for (size_t it = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; it < items; it += warps) {
+        const int b = (int)(it % r.batch);
+        const int t = (blk_lo + (int)(it / r.batch)) * B + j;
+        if (t >= m.T) continue;
+        const size_t at = (size_t)b * m.T + t;
+        const float *zz = m.logits + at * C;
+        const float *gg = r.noise + at * C;
+        float best = -INFINITY;
+        int bi = INT_MAX;
+        for (int c = lane; c < C; c += 32) {
+            const float v = zz[c] + gg[c];
+            if (v > best) { best = v; bi = c; }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(0xffffffffu, best, off);
+            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+            if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+        }
+        if (lane == 0) {
+            r.x[at] = (uint8_t)bi;
+            ((T *)m.a[0])[at] = from_f32<T>(m.lut[bi]);
+        }
+    }
+}
+
+// x_old = x and a_old[0] = a[0] (start of an outer iteration); or compare x with
+// x_old and raise change flags (end of an outer iteration).
+template <typename T>
+__device__ void jgs_copy_or_compare(const MadeDev &m, const RunArgs &r, bool compare, int parity)
+{
+    const size_t n = (size_t)r.batch * m.T;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        if (compare) {
+            if (r.x[i] != r.x_old[i]) note_change(r, parity, (int)(i / m.T), (int)(i % m.T));
+        } else {
+            r.x_old[i] = r.x[i];
+            ((T *)m.a_old[0])[i] = ((const T *)m.a[0])[i];
+        }
+    }
+}
+
+// ------------------------------------------------------------------ drivers
+template <typename T>
+__global__ void __launch_bounds__(NTHREADS) made_generic_kernel(const MadeDev m, const RunArgs r)
+{
+    __shared__ Smem s;
+    unsigned epoch = 0;
+    unsigned long long issued = 0, skipped = 0;
+    JsCtl *ctl = r.ctl;
+    T *acts[JS_MAXL + 1], *acts_old[JS_MAXL + 1];
+    for (int l = 0; l <= m.L; ++l) { acts[l] = (T *)m.a[l]; acts_old[l] = (T *)m.a_old[l]; }
+    const int T_ = m.T;
+    int status = JS_OK, iterations = 0, frontier = 0;
+    bool alive = true;
+
+#define BARRIER() do { if (!grid_barrier(ctl, epoch, r.spin_limit)) { alive = false; goto done; } } while (0)
+
+    if (r.kmode == KM_FORWARD) {
+        init_phase<T>(m, r, r.x_in);
+        BARRIER();
+        Win w = {0, T_, 0, T_};
+        if (!forward_pass<T>(s, m, r, acts, r.logits_out, w, epoch, issued, skipped)) { alive = false; goto done; }
+        iterations = 1;
+        goto done;
+    }
+
+    init_phase<T>(m, r, r.kmode == KM_SEQ ? (const uint8_t *)nullptr : r.init);
+    BARRIER();
+
+    if (r.kmode == KM_SEQ) {
+        // Eq. 1 in strict order: step t keeps position t of a forward pass.
+        for (int t = 0; t < T_; ++t) {
+            Win w;
+            if (r.seq_skip) w = Win{t - 1, t, t, t + 1};      // only the units that became computable
+            else w = Win{0, T_, 0, T_};                       // the whole network, every step
+            if (!forward_pass<T>(s, m, r, acts, m.logits, w, epoch, issued, skipped)) { alive = false; goto done; }
+            sample_phase<T>(m, r, m.logits, t, t + 1, false, 0);
+            BARRIER();
+            iterations++;
+        }
+        frontier = T_;
+        if (blockIdx.x == 0 && r.out_iters)
+            for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.out_iters[b] = 1;
+        goto done;
+    }
+
+    if (r.kmode == KM_JACOBI) {
+        // Algorithm 1 with per-sample stopping.
+        const int cap = (r.max_iters > 0 && r.max_iters < T_) ? r.max_iters : T_;
+        int fin_x = 0, fin_h = 0;
+        for (int k = 1;; ++k) {
+            const int p = k & 1;
+            Win w = r.frontier_skip ? Win{fin_h, T_, fin_x, T_} : Win{0, T_, 0, T_};
+            if (!forward_pass<T>(s, m, r, acts, m.logits, w, epoch, issued, skipped)) { alive = false; goto done; }
+            sample_phase<T>(m, r, m.logits, w.plo, T_, true, p);
+            BARRIER();
+            iterations++;
+            const int any = ld_volatile_i32(&ctl->agg_any[p]);
+            const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
+            book_samples(r, p, k, k == cap, false, true);
+            reset_other_parity(r, p);
+            fin_h = max(fin_h, fin_x);
+            fin_x = any ? max(fin_x + 1, min(mf + 1, T_)) : T_;
+            if (!any || k == cap) {
+                if (any && cap < T_) status = JS_NOT_CONVERGED;
+                break;
+            }
+        }
+        frontier = fin_x;
+        goto done;
+    }
+
+    if (r.kmode == KM_GS_JACOBI) {
+        // Algorithm 3: blocks in order, Jacobi inside the block.
+        const int B = r.block;
+        int fin_x = 0, fin_h = 0, tick = 0;
+        for (int a = 0; a < T_; a += B) {
+            const int bend = min(a + B, T_), len = bend - a;
+            const int cap = (r.max_iters > 0 && r.max_iters < len) ? r.max_iters : len;
+            int lo = a;                         // positions of the block below lo are settled
+            for (int k = 1;; ++k) {
+                const int p = (++tick) & 1;
+                Win w = r.frontier_skip ? Win{fin_h, bend - 1, lo, bend} : Win{0, T_, a, bend};
+                if (!forward_pass<T>(s, m, r, acts, m.logits, w, epoch, issued, skipped)) { alive = false; goto done; }
+                sample_phase<T>(m, r, m.logits, w.plo, bend, true, p);
+                BARRIER();
+                iterations++;
+                const int any = ld_volatile_i32(&ctl->agg_any[p]);
+                const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
+                const bool last = (!any || k == cap);
+                book_samples(r, p, k, k == cap, true, false);
+                reset_other_parity(r, p);
+                fin_h = max(fin_h, min(fin_x, bend - 1));
+                lo = any ? max(lo + 1, min(mf + 1, bend)) : bend;
+                fin_x = max(fin_x, lo);
+                if (last) {
+                    if (any && cap < len) status = JS_NOT_CONVERGED;
+                    break;
+                }
+            }
+            // positions < bend are never touched again: treat them as settled
+            fin_x = bend;
+            if (blockIdx.x == 0)
+                for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.smp_state[b] = 0;   // new block: nobody done
+            // (CTA 0 reads smp_state again only after the next barrier)
+        }
+        if (blockIdx.x == 0 && r.out_iters)
+            for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.out_iters[b] = r.smp_state[r.batch + b];
+        frontier = T_;
+        goto done;
+    }
+
+    if (r.kmode == KM_JACOBI_GS) {
+        // Algorithm 2: all blocks in parallel, a sequential sweep inside each.
+        const int B = r.block, M = (T_ + B - 1) / B;
+        const int cap = (r.max_iters > 0 && r.max_iters < M) ? r.max_iters : M;
+        int fin_x = 0, fin_h = 0;
+        for (int k = 1;; ++k) {
+            const int p = k & 1;
+            jgs_copy_or_compare<T>(m, r, false, p);
+            BARRIER();
+            // hidden activations of the previous outer iterate
+            Win w = r.frontier_skip ? Win{fin_h, T_, T_, T_} : Win{0, T_, T_, T_};
+            for (int l = 0; l < m.L; ++l) {
+                gemm_phase<T>(s, m, l, acts_old[l], acts_old[l + 1], nullptr, r.batch, w, issued, skipped);
+                BARRIER();
+            }
+            const int blk_lo = r.frontier_skip ? fin_x / B : 0;
+            const int jmax = min(B, T_);
+            for (int j = 0; j < jmax; ++j) {
+                if (j >= 1)
+                    for (int l = 0; l < m.L; ++l) {
+                        jgs_hidden_phase<T>(s, m, r, l, j, B, blk_lo);
+                        BARRIER();
+                    }
+                jgs_output_phase<T>(m, r, j, B, blk_lo);
+                BARRIER();
+                if (m.C > 1) {
+                    jgs_commit_phase<T>(m, r, j, B, blk_lo);
+                    BARRIER();
+                }
+                iterations++;
+            }
+            jgs_copy_or_compare<T>(m, r, true, p);
+            BARRIER();
+            const int any = ld_volatile_i32(&ctl->agg_any[p]);
+            const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
+            book_samples(r, p, k, k == cap, false, true);
+            reset_other_parity(r, p);
+            fin_h = max(fin_h, fin_x);
+            // after outer iteration k the first k blocks are final (proof of Prop. 2)
+            fin_x = any ? max(min(k * B, T_), min(mf + 1, T_)) : T_;
+            if (!any || k == cap) {
+                if (any && cap < M) status = JS_NOT_CONVERGED;
+                break;
+            }
+        }
+        frontier = fin_x;
+        goto done;
+    }
+
+done:
+#undef BARRIER
+    if (threadIdx.x == 0) {
+        atomicAdd(&ctl->tiles_issued, issued);
+        atomicAdd(&ctl->tiles_skipped, skipped);
+        if (blockIdx.x == 0) {
+            ctl->iterations = iterations;
+            ctl->frontier = frontier;
+            ctl->status = alive ? status : JS_ERR_TIMEOUT;
+        }
+    }
+}
+
+}  // namespace
+
+int js_made_generic_max_grid(int prec)
+{
+    int dev = 0, sms = 0, per_sm = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+    cudaError_t e = prec == JS_BF16
+        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, made_generic_kernel<__nv_bfloat16>, NTHREADS, 0)
+        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, made_generic_kernel<float>, NTHREADS, 0);
+    if (e != cudaSuccess || per_sm < 1) return -1;
+    return sms * per_sm;
+}
+
+int js_launch_made_generic(const MadeDev &m, const RunArgs &r, int grid, cudaStream_t stream)
+{
+    void *args[2] = {(void *)&m, (void *)&r};
+    const void *fn = m.prec == JS_BF16 ? (const void *)made_generic_kernel<__nv_bfloat16>
+                                       : (const void *)made_generic_kernel<float>;
+    cudaError_t e = cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(NTHREADS), args, 0, stream);
+    return e == cudaSuccess ? 0 : (int)e;
+}

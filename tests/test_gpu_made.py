@@ -1,0 +1,239 @@
+"""Parity of the CUDA masked-MLP sampler with the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from parity import check_samples, logits_close
+
+pytestmark = pytest.mark.gpu
+
+
+def pkg():
+    import __graft_entry__ as ge
+    ge.build()
+    import paper_2002_03629_b200 as p
+    return p
+
+
+class Case:
+    """Arrays, oracle model and CUDA model of one workload."""
+
+    def __init__(self, cfg, salt=0, path=None):
+        p = pkg()
+        self.p, self.cfg = p, cfg
+        self.W, self.b = si.made_weights(cfg, salt)
+        self.lut = si.made_lut(cfg)
+        self.noise = si.draw_noise(cfg, salt=salt)
+        self.orc = oracle.from_config(cfg, self.W, self.b, self.lut)
+        self.model = p.Model.from_config(cfg, self.W, self.b, self.lut)
+        if path is not None:
+            self.model.set_option(p.JS_OPT_PATH, path)
+        self.d_noise = torch.from_numpy(self.noise).cuda()
+        self.nk = cfg.noise_kind
+        self._xstar = None
+
+    @property
+    def xstar(self):
+        if self._xstar is None:
+            self._xstar = self.orc.sequential_batch(self.noise, self.nk, threads=8)
+        return self._xstar
+
+    def run(self, mode, block=0, max_iters=0, init=None):
+        cfg, p = self.cfg, self.p
+        out = torch.full((cfg.batch, cfg.D), 255, dtype=torch.uint8, device="cuda")
+        iters = torch.full((cfg.batch,), -1, dtype=torch.int32, device="cuda")
+        d_init = None if init is None else torch.from_numpy(init).cuda()
+        rc = p.jacobi_sample(self.model, self.d_noise, self.nk, d_init, mode, block, max_iters, out, iters)
+        return rc, out.cpu().numpy(), iters.cpu().numpy()
+
+    def oracle_counts(self, mode, block=0, max_iters=0, init=None, samples=None):
+        p, o = self.p, self.orc
+        samples = range(self.cfg.batch) if samples is None else samples
+        xs, its = [], []
+        for s in samples:
+            i0 = None if init is None else init[s]
+            if mode == p.JS_JACOBI:
+                x, it, _, _ = o.jacobi(self.noise[s], self.nk, i0, max_iters)
+            elif mode == p.JS_GS_JACOBI:
+                x, it, _ = o.gs_jacobi(self.noise[s], self.nk, block, i0, max_iters)
+            elif mode == p.JS_JACOBI_GS:
+                x, it, _ = o.jacobi_gs(self.noise[s], self.nk, block, i0, max_iters)
+            else:
+                x, it = o.gauss_seidel(self.noise[s], self.nk, i0), 1
+            xs.append(x)
+            its.append(it)
+        return np.stack(xs), np.array(its, dtype=np.int32)
+
+    def check(self, mode, block=0, init=None, expect_rc=0):
+        rc, x, it = self.run(mode, block, 0, init)
+        assert rc == expect_rc
+        audit = check_samples(self.orc, x, self.xstar, self.noise, self.nk)
+        _, it_ref = self.oracle_counts(mode, block, 0, init)
+        clean = np.setdiff1d(np.arange(self.cfg.batch), audit["excused_samples"])
+        np.testing.assert_array_equal(it[clean], it_ref[clean])
+        return audit, it, it_ref
+
+
+TINY = si.CONFIGS["made_tiny"]
+BIN = si.scaled(si.CONFIGS["made_784"], D=200, H=(192, 160), batch=70)        # ragged tiles
+CAT = si.scaled(si.CONFIGS["made_cat"], D=24, H=(128, 96), batch=9)
+CHAIN = si.scaled(si.CONFIGS["made_4096"], D=256, H=(256, 256, 256, 256), batch=130, w_var_scale=4.0)
+
+CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN}
+_cache = {}
+
+
+def case(name, path=1):
+    key = (name, path)
+    if key not in _cache:
+        _cache[key] = Case(CASES[name], path=path)
+    return _cache[key]
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_logits_match_oracle(name):
+    c = case(name)
+    cfg, p = c.cfg, c.p
+    x = si.random_init(cfg, salt=5)
+    logits = torch.empty((cfg.batch, cfg.D, cfg.C), dtype=torch.float32, device="cuda")
+    assert p.js_forward_logits(c.model, torch.from_numpy(x).cuda(), logits) == 0
+    got = logits.cpu().numpy()
+    n = min(cfg.batch, 6)
+    ref = np.stack([c.orc.forward_logits(x[s]) for s in range(n)])
+    rel = 1e-5 if cfg.prec == si.PREC_F32 else 2e-2
+    err, ok = logits_close(got[:n], ref, rel)
+    assert ok, err
+
+
+@pytest.mark.parametrize("name", list(CASES))
+@pytest.mark.parametrize("skip", [1, 0])
+def test_jacobi_matches_sequential_and_counts(name, skip):
+    c = case(name)
+    c.model.set_option(c.p.JS_OPT_FRONTIER_SKIP, skip)
+    try:
+        c.check(c.p.JS_JACOBI)
+        c.check(c.p.JS_JACOBI, init=si.random_init(c.cfg, salt=1))
+    finally:
+        c.model.set_option(c.p.JS_OPT_FRONTIER_SKIP, 1)
+
+
+@pytest.mark.parametrize("name", list(CASES))
+@pytest.mark.parametrize("seq_skip", [0, 1])
+def test_sequential_and_gauss_seidel(name, seq_skip):
+    c = case(name)
+    p, cfg = c.p, c.cfg
+    c.model.set_option(p.JS_OPT_SEQ_SKIP, seq_skip)
+    try:
+        out = torch.empty((cfg.batch, cfg.D), dtype=torch.uint8, device="cuda")
+        assert p.sequential_sample(c.model, c.d_noise, c.nk, out) == 0
+        check_samples(c.orc, out.cpu().numpy(), c.xstar, c.noise, c.nk)
+        rc, x, it = c.run(p.JS_GAUSS_SEIDEL, init=si.random_init(cfg, salt=2))
+        assert rc == 0 and np.all(it == 1)
+        check_samples(c.orc, x, c.xstar, c.noise, c.nk)
+    finally:
+        c.model.set_option(p.JS_OPT_SEQ_SKIP, 0)
+
+
+@pytest.mark.parametrize("name,blocks", [("tiny", (1, 4, 5, 16)), ("bin", (64, 30)), ("cat", (8, 5)),
+                                         ("chain", (32, 64))])
+@pytest.mark.parametrize("skip", [1, 0])
+def test_hybrids(name, blocks, skip):
+    c = case(name)
+    p = c.p
+    c.model.set_option(p.JS_OPT_FRONTIER_SKIP, skip)
+    try:
+        for B in blocks:
+            for init in (None, si.random_init(c.cfg, salt=3)):
+                c.check(p.JS_GS_JACOBI, B, init)
+                c.check(p.JS_JACOBI_GS, B, init)
+    finally:
+        c.model.set_option(p.JS_OPT_FRONTIER_SKIP, 1)
+
+
+@pytest.mark.parametrize("name", ["bin", "chain"])
+def test_max_iters_returns_last_iterate(name):
+    c = case(name)
+    p = c.p
+    _, it_full = c.oracle_counts(p.JS_JACOBI)
+    k = max(2, int(it_full.max()) // 2)
+    rc, x, it = c.run(p.JS_JACOBI, max_iters=k)
+    x_ref, it_ref = c.oracle_counts(p.JS_JACOBI, max_iters=k)
+    assert rc == (p.JS_NOT_CONVERGED if it_full.max() > k else 0)
+    exact = np.all(x == x_ref, axis=1)
+    assert exact.mean() > 0.9                      # near-ties may differ; the bulk must be identical
+    np.testing.assert_array_equal(it[exact], it_ref[exact])
+
+
+def test_examples_of_section_4_on_device():
+    """Markov chain (Example 3): T iterations; independent chain (Example 1): one plus the confirmation."""
+    p = pkg()
+    T, c0 = 40, 64.0
+    H = T - 1
+    W0 = np.zeros((H, T), np.float32)
+    W1 = np.zeros((T, H), np.float32)
+    for j in range(H):
+        W0[j, j] = 1.0
+        W1[j + 1, j] = c0
+    b1 = np.full(T, -c0 / 2, np.float32)
+    b1[0] = c0
+    cfg = si.MadeConfig("ex3", 41, D=T, C=1, H=(H,), act=si.ACT_RELU, prec=si.PREC_F32, batch=5,
+                        noise_kind=si.NOISE_LOGISTIC)
+    noise = si.draw_noise(cfg)
+    lut = np.array([0, 1], np.float32)
+    for W, expect in (([W0, W1], T), ([W0 * 0, W1 * 0], 2)):
+        m = p.Model.made(T, 1, [H], p.JS_ACT_RELU, p.JS_F32, W, [np.zeros(H, np.float32), b1], lut, cfg.batch)
+        out = torch.empty((cfg.batch, T), dtype=torch.uint8, device="cuda")
+        iters = torch.empty((cfg.batch,), dtype=torch.int32, device="cuda")
+        assert p.jacobi_sample(m, torch.from_numpy(noise).cuda(), si.NOISE_LOGISTIC, None, p.JS_JACOBI, 0, 0, out,
+                               iters) == 0
+        assert np.all(iters.cpu().numpy() == expect)
+        if expect == T:
+            assert np.all(out.cpu().numpy() == 1)
+        m.close()
+
+
+def test_argument_errors():
+    c = case("tiny")
+    p, cfg = c.p, c.cfg
+    out = torch.empty((cfg.batch, cfg.D), dtype=torch.uint8, device="cuda")
+    lib = p.load_library()
+    h = c.model._h
+    s = torch.cuda.current_stream().cuda_stream
+    assert lib.jacobi_sample(h, cfg.batch, None, c.nk, None, 0, 0, 0, out.data_ptr(), None, s) == p.JS_ERR_ARG
+    assert lib.jacobi_sample(h, cfg.batch + 1, c.d_noise.data_ptr(), c.nk, None, 0, 0, 0, out.data_ptr(), None,
+                             s) == p.JS_ERR_ARG
+    assert lib.jacobi_sample(h, cfg.batch, c.d_noise.data_ptr(), c.nk, None, 7, 0, 0, out.data_ptr(), None,
+                             s) == p.JS_ERR_ARG
+    assert lib.jacobi_sample(h, cfg.batch, c.d_noise.data_ptr(), p.JS_NOISE_GUMBEL, None, 0, 0, 0, out.data_ptr(),
+                             None, s) == p.JS_ERR_ARG
+    assert lib.jacobi_sample(h, cfg.batch, c.d_noise.data_ptr(), c.nk, None, p.JS_GS_JACOBI, 0, 0, out.data_ptr(),
+                             None, s) == p.JS_ERR_ARG
+    assert lib.jacobi_sample(None, cfg.batch, c.d_noise.data_ptr(), c.nk, None, 0, 0, 0, out.data_ptr(), None,
+                             s) == p.JS_ERR_ARG
+
+
+def test_bounded_wait_reports_timeout_and_model_stays_usable():
+    """With a spin limit of zero the first grid barrier gives up: the call returns
+    JS_ERR_TIMEOUT instead of hanging, and the next call works again."""
+    c = case("bin")
+    p = c.p
+    c.model.set_option(p.JS_OPT_SPIN_LIMIT, 0)
+    try:
+        with pytest.raises(p.JsError) as e:
+            c.run(p.JS_JACOBI)
+        assert e.value.code == p.JS_ERR_TIMEOUT
+    finally:
+        c.model.set_option(p.JS_OPT_SPIN_LIMIT, 1 << 22)
+    c.check(p.JS_JACOBI)
+
+
+def test_batch_of_one_and_aliasing_init():
+    c = case("bin")
+    p, cfg = c.p, c.cfg
+    init = si.random_init(cfg, salt=4)
+    buf = torch.from_numpy(init[:1].copy()).cuda()
+    rc = p.jacobi_sample(c.model, c.d_noise[:1].contiguous(), c.nk, buf, p.JS_JACOBI, 0, 0, buf, None)
+    assert rc == 0
+    check_samples(c.orc, buf.cpu().numpy(), c.xstar[:1], c.noise[:1], c.nk)
