@@ -189,6 +189,12 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
 
     int used_path = 1;
     int rc_launch;
+    // the tensor-core epilogues use 16-byte vector accesses on the caller's buffers
+    const bool aligned = (((uintptr_t)r.noise | (uintptr_t)r.x | (uintptr_t)r.logits_out) & 15u) == 0;
+    if (m->tc_ok && m->opt_path == 0 && r.kmode != KM_JACOBI_GS && aligned) {
+        used_path = 0;
+        rc_launch = js_launch_made_tc(m, r, st);
+    } else {
     if (m->max_grid_generic <= 0) m->max_grid_generic = js_made_generic_max_grid(v.prec);
     if (m->max_grid_generic <= 0) {
         snprintf(g_cuda_err, sizeof g_cuda_err, "occupancy query failed");
@@ -201,6 +207,7 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
         const long long elems = ((long long)r.batch * v.T * (v.C > 1 ? 32 : 1) + 255) / 256;
         const int grid = (int)std::min<long long>(m->max_grid_generic, std::max(tiles, elems));
         rc_launch = js_launch_made_generic(v, r, std::max(grid, 1), st);
+    }
     }
     if (rc_launch != 0) {
         snprintf(g_cuda_err, sizeof g_cuda_err, "kernel launch: %s", cudaGetErrorString((cudaError_t)rc_launch));
@@ -248,6 +255,7 @@ int js_made_create(const js_made_desc *d, js_model **out)
     m->max_batch = d->max_batch;
     int rc = made_build(m, d);
     if (rc == JS_OK) rc = common_scratch(m, d->T);
+    if (rc == JS_OK && js_tc_prepare(m) < 0) rc = JS_ERR_CUDA;
     if (rc != JS_OK) { js_model_destroy(m); return rc; }
     *out = m;
     return JS_OK;

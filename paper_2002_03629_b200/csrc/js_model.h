@@ -1,8 +1,26 @@
 // Host-side model object behind the opaque js_model handle.
 #pragma once
+#include <cuda.h>
+
 #include <vector>
 
 #include "js_common.cuh"
+
+// Tensor-core view of a masked MLP: per layer the output-tile width, the tile
+// metadata (last live K block, smallest / largest degree) and the TMA descriptors.
+struct TcLayer {
+    const int *kb_end;
+    const int *dmin;
+    const int *dmax;
+    int bn;
+    int nt;
+};
+struct TcDev {
+    const CUtensorMap *tmA;      // [L+1] activations a[l], box 64 x 128
+    const CUtensorMap *tmW;      // [L+1] masked weights W[l], box 64 x bn
+    TcLayer lay[JS_MAXL + 1];
+    int stage_bytes, n_stages;
+};
 
 struct js_model {
     int kind = 0;                 // 0 masked MLP, 1 masked-conv stack
@@ -17,5 +35,10 @@ struct js_model {
     uint8_t *x_old = nullptr, *x_tmp = nullptr;
     int opt_frontier_skip = 1, opt_seq_skip = 0, opt_spin_limit = 1 << 22, opt_path = 0, opt_compact = 1;
     int max_grid_generic = 0;
+    TcDev tc{};
+    int tc_ok = 0, tc_max_grid = 0;
     js_stats stats{};
 };
+
+int js_tc_prepare(js_model *m);
+int js_launch_made_tc(const js_model *m, const RunArgs &r, cudaStream_t stream);

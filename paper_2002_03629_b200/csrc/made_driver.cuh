@@ -1,0 +1,209 @@
+// Device-side solver loops shared by the masked-MLP kernels.  An engine supplies
+// the phases (grid barrier, initialisation, one windowed forward pass with the
+// sampling step); the driver is the control logic of Algorithms 1-3 and of the
+// strict feedforward order, executed identically by every thread of every CTA.
+//
+// Window bookkeeping.  fin_x = number of leading positions of the current
+// iterate known to be final; fin_h = hidden units of degree <= fin_h hold their
+// final values.  The proof of Proposition 1 gives fin_x >= k after k Jacobi
+// iterations; more sharply, if an iteration left positions < j unchanged they
+// solve their equations, so positions <= j are final.  A forward pass on an
+// iterate with fin_x final positions makes hidden units of degree <= fin_x final.
+#pragma once
+#include <limits.h>
+
+#include "js_common.cuh"
+
+struct Win {
+    int hdeg_lo;   // hidden units of degree <= hdeg_lo are final: not recomputed
+    int hdeg_hi;   // hidden units of degree >  hdeg_hi are not needed yet
+    int plo, phi;  // output positions [plo, phi) are sampled and committed
+    int olo, ohi;  // output positions [olo, ohi) are computed (>= the committed range)
+};
+
+__device__ __forceinline__ Win make_win(int hlo, int hhi, int plo, int phi)
+{
+    Win w = {hlo, hhi, plo, phi, plo, phi};
+    return w;
+}
+
+__device__ __forceinline__ void note_change(const RunArgs &r, int parity, int b, int d)
+{
+    atomicOr(&r.smp_changed[parity * r.batch + b], 1);
+    atomicMin(&r.ctl->agg_minfirst[parity], d);
+    atomicOr(&r.ctl->agg_any[parity], 1);
+}
+
+// After the barrier that ends an iteration: CTA 0 clears the other parity's flags.
+// Safe because every CTA read that parity before it passed at least one later
+// barrier, and nobody writes it again before at least one more barrier.
+__device__ __forceinline__ void reset_other_parity(const RunArgs &r, int parity)
+{
+    if (blockIdx.x != 0) return;
+    const int o = parity ^ 1;
+    for (int i = threadIdx.x; i < r.batch; i += blockDim.x) r.smp_changed[o * r.batch + i] = 0;
+    if (threadIdx.x == 0) {
+        r.ctl->agg_any[o] = 0;
+        r.ctl->agg_minfirst[o] = INT_MAX;
+    }
+}
+
+// CTA 0: a sample whose iterate did not change (or that hit the cap) stops counting.
+__device__ __forceinline__ void book_samples(const RunArgs &r, int parity, int k, bool at_cap, bool add,
+                                             bool final_write)
+{
+    if (blockIdx.x != 0) return;
+    int *done = r.smp_state, *count = r.smp_state + r.batch;
+    for (int b = threadIdx.x; b < r.batch; b += blockDim.x) {
+        if (!done[b] && (r.smp_changed[parity * r.batch + b] == 0 || at_cap)) {
+            done[b] = 1;
+            count[b] = add ? count[b] + k : k;
+            if (final_write && r.out_iters) r.out_iters[b] = count[b];
+        }
+    }
+}
+
+struct DriverResult {
+    int status, iterations, frontier;
+    bool alive;
+};
+
+template <class E>
+__device__ DriverResult made_driver(E &e, const MadeDev &m, const RunArgs &r)
+{
+    DriverResult res = {JS_OK, 0, 0, true};
+    JsCtl *ctl = r.ctl;
+    const int T_ = m.T;
+
+    if (r.kmode == KM_FORWARD) {
+        e.init(r.x_in);
+        if (!e.barrier()) { res.alive = false; return res; }
+        if (!e.forward_logits(r.logits_out)) { res.alive = false; return res; }
+        res.iterations = 1;
+        return res;
+    }
+
+    e.init(r.kmode == KM_SEQ ? (const uint8_t *)nullptr : r.init);
+    if (!e.barrier()) { res.alive = false; return res; }
+
+    if (r.kmode == KM_SEQ) {
+        // Eq. 1 in strict order: step t keeps position t of a forward pass.
+        for (int t = 0; t < T_; ++t) {
+            Win w = make_win(0, T_, t, t + 1);
+            if (r.seq_skip) w.hdeg_lo = t - 1, w.hdeg_hi = t;     // only the units that became computable
+            else w.olo = 0, w.ohi = T_;                           // the whole network, every step
+            if (!e.step(w, false, 0)) { res.alive = false; return res; }
+            res.iterations++;
+        }
+        res.frontier = T_;
+        if (blockIdx.x == 0 && r.out_iters)
+            for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.out_iters[b] = 1;
+        return res;
+    }
+
+    if (r.kmode == KM_JACOBI) {
+        // Algorithm 1 with per-sample stopping.
+        const int cap = (r.max_iters > 0 && r.max_iters < T_) ? r.max_iters : T_;
+        int fin_x = 0, fin_h = 0;
+        for (int k = 1;; ++k) {
+            const int p = k & 1;
+            const Win w = r.frontier_skip ? make_win(fin_h, T_, fin_x, T_) : make_win(0, T_, 0, T_);
+            if (!e.step(w, true, p)) { res.alive = false; return res; }
+            res.iterations++;
+            const int any = ld_volatile_i32(&ctl->agg_any[p]);
+            const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
+            book_samples(r, p, k, k == cap, false, true);
+            reset_other_parity(r, p);
+            fin_h = max(fin_h, fin_x);
+            fin_x = any ? max(fin_x + 1, min(mf + 1, T_)) : T_;
+            if (!any || k == cap) {
+                if (any && cap < T_) res.status = JS_NOT_CONVERGED;
+                break;
+            }
+        }
+        res.frontier = fin_x;
+        return res;
+    }
+
+    if (r.kmode == KM_GS_JACOBI) {
+        // Algorithm 3: blocks in order, Jacobi inside the block.
+        const int B = r.block;
+        int fin_x = 0, fin_h = 0, tick = 0;
+        for (int a = 0; a < T_; a += B) {
+            const int bend = min(a + B, T_), len = bend - a;
+            const int cap = (r.max_iters > 0 && r.max_iters < len) ? r.max_iters : len;
+            int lo = a;                         // positions of the block below lo are settled
+            for (int k = 1;; ++k) {
+                const int p = (++tick) & 1;
+                const Win w = r.frontier_skip ? make_win(fin_h, bend - 1, lo, bend) : make_win(0, T_, a, bend);
+                if (!e.step(w, true, p)) { res.alive = false; return res; }
+                res.iterations++;
+                const int any = ld_volatile_i32(&ctl->agg_any[p]);
+                const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
+                book_samples(r, p, k, k == cap, true, false);
+                reset_other_parity(r, p);
+                fin_h = max(fin_h, min(fin_x, bend - 1));
+                lo = any ? max(lo + 1, min(mf + 1, bend)) : bend;
+                fin_x = max(fin_x, lo);
+                if (!any || k == cap) {
+                    if (any && cap < len) res.status = JS_NOT_CONVERGED;
+                    break;
+                }
+            }
+            fin_x = bend;      // positions < bend are never touched again: settled
+            if (blockIdx.x == 0)   // new block: nobody is done (same threads wrote these entries)
+                for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.smp_state[b] = 0;
+        }
+        if (blockIdx.x == 0 && r.out_iters)
+            for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.out_iters[b] = r.smp_state[r.batch + b];
+        res.frontier = T_;
+        return res;
+    }
+
+    if (r.kmode == KM_JACOBI_GS) {
+        if constexpr (E::has_jgs) {
+            // Algorithm 2: all blocks in parallel, a sequential sweep inside each.
+            const int B = r.block, M = (T_ + B - 1) / B;
+            const int cap = (r.max_iters > 0 && r.max_iters < M) ? r.max_iters : M;
+            int fin_x = 0, fin_h = 0;
+            for (int k = 1;; ++k) {
+                const int p = k & 1;
+                if (!e.jgs_outer(p, r.frontier_skip ? fin_h : 0, r.frontier_skip ? fin_x / B : 0, res.iterations)) {
+                    res.alive = false;
+                    return res;
+                }
+                const int any = ld_volatile_i32(&ctl->agg_any[p]);
+                const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
+                book_samples(r, p, k, k == cap, false, true);
+                reset_other_parity(r, p);
+                fin_h = max(fin_h, fin_x);
+                // after outer iteration k the first k blocks are final (proof of Prop. 2)
+                fin_x = any ? max(min(k * B, T_), min(mf + 1, T_)) : T_;
+                if (!any || k == cap) {
+                    if (any && cap < M) res.status = JS_NOT_CONVERGED;
+                    break;
+                }
+            }
+            res.frontier = fin_x;
+        } else {
+            res.status = JS_ERR_UNSUPPORTED;
+        }
+        return res;
+    }
+    res.status = JS_ERR_ARG;
+    return res;
+}
+
+__device__ __forceinline__ void driver_finish(const RunArgs &r, const DriverResult &res, unsigned long long issued,
+                                              unsigned long long skipped)
+{
+    if (threadIdx.x == 0) {
+        atomicAdd(&r.ctl->tiles_issued, issued);
+        atomicAdd(&r.ctl->tiles_skipped, skipped);
+        if (blockIdx.x == 0) {
+            r.ctl->iterations = res.iterations;
+            r.ctl->frontier = res.frontier;
+            r.ctl->status = res.alive ? res.status : JS_ERR_TIMEOUT;
+        }
+    }
+}

@@ -11,18 +11,13 @@
 #include <limits.h>
 
 #include "js_common.cuh"
+#include "made_driver.cuh"
 
 namespace {
 
 constexpr int GT = JS_GT;      // 64x64 output tile
 constexpr int KC = 32;         // k chunk staged in shared memory
 constexpr int NTHREADS = 256;
-
-struct Win {
-    int hdeg_lo;   // hidden units of degree <= hdeg_lo are final: not recomputed
-    int hdeg_hi;   // hidden units of degree >  hdeg_hi are not needed yet
-    int plo, phi;  // output positions [plo, phi)
-};
 
 struct Smem {
     float As[KC][GT + 4];
@@ -88,7 +83,7 @@ __device__ void gemm_phase(Smem &s, const MadeDev &m, int l, const T *Asrc, T *o
         const int tn = tile / mt, tm = tile % mt;
         const int dmin = m.t_dmin[l][tn], dmax = m.t_dmax[l][tn];
         bool live;
-        if (is_out) live = (dmax - 1 >= w.plo) && (dmin - 1 < w.phi);
+        if (is_out) live = (dmax - 1 >= w.olo) && (dmin - 1 < w.ohi);
         else live = (dmax > w.hdeg_lo) && (dmin <= w.hdeg_hi);
         if (!live) { if (threadIdx.x == 0) skipped++; continue; }
         if (threadIdx.x == 0) issued++;
@@ -133,13 +128,6 @@ __device__ void init_phase(const MadeDev &m, const RunArgs &r, const uint8_t *sr
             r.ctl->agg_minfirst[0] = r.ctl->agg_minfirst[1] = INT_MAX;
         }
     }
-}
-
-__device__ __forceinline__ void note_change(const RunArgs &r, int parity, int b, int d)
-{
-    atomicOr(&r.smp_changed[parity * r.batch + b], 1);
-    atomicMin(&r.ctl->agg_minfirst[parity], d);
-    atomicOr(&r.ctl->agg_any[parity], 1);
 }
 
 // Sample positions [plo, phi) of every sample from the logits scratch, compare
@@ -188,32 +176,6 @@ __device__ void sample_phase(const MadeDev &m, const RunArgs &r, const float *z,
             r.x[at] = (uint8_t)bi;
             a0[at] = from_f32<T>(m.lut[bi]);
             if (flag) note_change(r, parity, b, d);
-        }
-    }
-}
-
-// After the barrier that ends an iteration: CTA 0 clears the other parity's flags.
-__device__ void reset_other_parity(const RunArgs &r, int parity)
-{
-    if (blockIdx.x != 0) return;
-    const int o = parity ^ 1;
-    for (int i = threadIdx.x; i < r.batch; i += blockDim.x) r.smp_changed[o * r.batch + i] = 0;
-    if (threadIdx.x == 0) {
-        r.ctl->agg_any[o] = 0;
-        r.ctl->agg_minfirst[o] = INT_MAX;
-    }
-}
-
-// CTA 0: a sample whose iterate did not change (or that hit the cap) stops counting.
-__device__ void book_samples(const RunArgs &r, int parity, int k, bool at_cap, bool add, bool final_write)
-{
-    if (blockIdx.x != 0) return;
-    int *done = r.smp_state, *count = r.smp_state + r.batch;
-    for (int b = threadIdx.x; b < r.batch; b += blockDim.x) {
-        if (!done[b] && (r.smp_changed[parity * r.batch + b] == 0 || at_cap)) {
-            done[b] = 1;
-            count[b] = add ? count[b] + k : k;
-            if (final_write && r.out_iters) r.out_iters[b] = count[b];
         }
     }
 }
@@ -378,177 +340,73 @@ __device__ void jgs_copy_or_compare(const MadeDev &m, const RunArgs &r, bool com
     }
 }
 
-// ------------------------------------------------------------------ drivers
+// ------------------------------------------------------------------ engine
 template <typename T>
-__global__ void __launch_bounds__(NTHREADS) made_generic_kernel(const MadeDev m, const RunArgs r)
-{
-    __shared__ Smem s;
+struct GenericEngine {
+    static constexpr bool has_jgs = true;
+    Smem &s;
+    const MadeDev &m;
+    const RunArgs &r;
     unsigned epoch = 0;
     unsigned long long issued = 0, skipped = 0;
-    JsCtl *ctl = r.ctl;
     T *acts[JS_MAXL + 1], *acts_old[JS_MAXL + 1];
-    for (int l = 0; l <= m.L; ++l) { acts[l] = (T *)m.a[l]; acts_old[l] = (T *)m.a_old[l]; }
-    const int T_ = m.T;
-    int status = JS_OK, iterations = 0, frontier = 0;
-    bool alive = true;
 
-#define BARRIER() do { if (!grid_barrier(ctl, epoch, r.spin_limit)) { alive = false; goto done; } } while (0)
-
-    if (r.kmode == KM_FORWARD) {
-        init_phase<T>(m, r, r.x_in);
-        BARRIER();
-        Win w = {0, T_, 0, T_};
-        if (!forward_pass<T>(s, m, r, acts, r.logits_out, w, epoch, issued, skipped)) { alive = false; goto done; }
-        iterations = 1;
-        goto done;
+    __device__ GenericEngine(Smem &s_, const MadeDev &m_, const RunArgs &r_) : s(s_), m(m_), r(r_)
+    {
+        for (int l = 0; l <= m.L; ++l) { acts[l] = (T *)m.a[l]; acts_old[l] = (T *)m.a_old[l]; }
     }
-
-    init_phase<T>(m, r, r.kmode == KM_SEQ ? (const uint8_t *)nullptr : r.init);
-    BARRIER();
-
-    if (r.kmode == KM_SEQ) {
-        // Eq. 1 in strict order: step t keeps position t of a forward pass.
-        for (int t = 0; t < T_; ++t) {
-            Win w;
-            if (r.seq_skip) w = Win{t - 1, t, t, t + 1};      // only the units that became computable
-            else w = Win{0, T_, 0, T_};                       // the whole network, every step
-            if (!forward_pass<T>(s, m, r, acts, m.logits, w, epoch, issued, skipped)) { alive = false; goto done; }
-            sample_phase<T>(m, r, m.logits, t, t + 1, false, 0);
-            BARRIER();
+    __device__ bool barrier() { return grid_barrier(r.ctl, epoch, r.spin_limit); }
+    __device__ void init(const uint8_t *src) { init_phase<T>(m, r, src); }
+    __device__ bool forward_logits(float *zout)
+    {
+        const Win w = make_win(0, m.T, 0, m.T);
+        return forward_pass<T>(s, m, r, acts, zout, w, epoch, issued, skipped);
+    }
+    __device__ bool step(const Win &w, bool flag, int parity)
+    {
+        if (!forward_pass<T>(s, m, r, acts, m.logits, w, epoch, issued, skipped)) return false;
+        sample_phase<T>(m, r, m.logits, w.plo, w.phi, flag, parity);
+        return barrier();
+    }
+    // one outer iteration of Algorithm 2
+    __device__ bool jgs_outer(int parity, int fin_h, int blk_lo, int &iterations)
+    {
+        const int B = r.block, T_ = m.T;
+        jgs_copy_or_compare<T>(m, r, false, parity);
+        if (!barrier()) return false;
+        // hidden activations of the previous outer iterate
+        const Win w = make_win(fin_h, T_, T_, T_);
+        for (int l = 0; l < m.L; ++l) {
+            gemm_phase<T>(s, m, l, acts_old[l], acts_old[l + 1], nullptr, r.batch, w, issued, skipped);
+            if (!barrier()) return false;
+        }
+        const int jmax = min(B, T_);
+        for (int j = 0; j < jmax; ++j) {
+            if (j >= 1)
+                for (int l = 0; l < m.L; ++l) {
+                    jgs_hidden_phase<T>(s, m, r, l, j, B, blk_lo);
+                    if (!barrier()) return false;
+                }
+            jgs_output_phase<T>(m, r, j, B, blk_lo);
+            if (!barrier()) return false;
+            if (m.C > 1) {
+                jgs_commit_phase<T>(m, r, j, B, blk_lo);
+                if (!barrier()) return false;
+            }
             iterations++;
         }
-        frontier = T_;
-        if (blockIdx.x == 0 && r.out_iters)
-            for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.out_iters[b] = 1;
-        goto done;
+        jgs_copy_or_compare<T>(m, r, true, parity);
+        return barrier();
     }
+};
 
-    if (r.kmode == KM_JACOBI) {
-        // Algorithm 1 with per-sample stopping.
-        const int cap = (r.max_iters > 0 && r.max_iters < T_) ? r.max_iters : T_;
-        int fin_x = 0, fin_h = 0;
-        for (int k = 1;; ++k) {
-            const int p = k & 1;
-            Win w = r.frontier_skip ? Win{fin_h, T_, fin_x, T_} : Win{0, T_, 0, T_};
-            if (!forward_pass<T>(s, m, r, acts, m.logits, w, epoch, issued, skipped)) { alive = false; goto done; }
-            sample_phase<T>(m, r, m.logits, w.plo, T_, true, p);
-            BARRIER();
-            iterations++;
-            const int any = ld_volatile_i32(&ctl->agg_any[p]);
-            const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
-            book_samples(r, p, k, k == cap, false, true);
-            reset_other_parity(r, p);
-            fin_h = max(fin_h, fin_x);
-            fin_x = any ? max(fin_x + 1, min(mf + 1, T_)) : T_;
-            if (!any || k == cap) {
-                if (any && cap < T_) status = JS_NOT_CONVERGED;
-                break;
-            }
-        }
-        frontier = fin_x;
-        goto done;
-    }
-
-    if (r.kmode == KM_GS_JACOBI) {
-        // Algorithm 3: blocks in order, Jacobi inside the block.
-        const int B = r.block;
-        int fin_x = 0, fin_h = 0, tick = 0;
-        for (int a = 0; a < T_; a += B) {
-            const int bend = min(a + B, T_), len = bend - a;
-            const int cap = (r.max_iters > 0 && r.max_iters < len) ? r.max_iters : len;
-            int lo = a;                         // positions of the block below lo are settled
-            for (int k = 1;; ++k) {
-                const int p = (++tick) & 1;
-                Win w = r.frontier_skip ? Win{fin_h, bend - 1, lo, bend} : Win{0, T_, a, bend};
-                if (!forward_pass<T>(s, m, r, acts, m.logits, w, epoch, issued, skipped)) { alive = false; goto done; }
-                sample_phase<T>(m, r, m.logits, w.plo, bend, true, p);
-                BARRIER();
-                iterations++;
-                const int any = ld_volatile_i32(&ctl->agg_any[p]);
-                const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
-                const bool last = (!any || k == cap);
-                book_samples(r, p, k, k == cap, true, false);
-                reset_other_parity(r, p);
-                fin_h = max(fin_h, min(fin_x, bend - 1));
-                lo = any ? max(lo + 1, min(mf + 1, bend)) : bend;
-                fin_x = max(fin_x, lo);
-                if (last) {
-                    if (any && cap < len) status = JS_NOT_CONVERGED;
-                    break;
-                }
-            }
-            // positions < bend are never touched again: treat them as settled
-            fin_x = bend;
-            if (blockIdx.x == 0)
-                for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.smp_state[b] = 0;   // new block: nobody done
-            // (CTA 0 reads smp_state again only after the next barrier)
-        }
-        if (blockIdx.x == 0 && r.out_iters)
-            for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.out_iters[b] = r.smp_state[r.batch + b];
-        frontier = T_;
-        goto done;
-    }
-
-    if (r.kmode == KM_JACOBI_GS) {
-        // Algorithm 2: all blocks in parallel, a sequential sweep inside each.
-        const int B = r.block, M = (T_ + B - 1) / B;
-        const int cap = (r.max_iters > 0 && r.max_iters < M) ? r.max_iters : M;
-        int fin_x = 0, fin_h = 0;
-        for (int k = 1;; ++k) {
-            const int p = k & 1;
-            jgs_copy_or_compare<T>(m, r, false, p);
-            BARRIER();
-            // hidden activations of the previous outer iterate
-            Win w = r.frontier_skip ? Win{fin_h, T_, T_, T_} : Win{0, T_, T_, T_};
-            for (int l = 0; l < m.L; ++l) {
-                gemm_phase<T>(s, m, l, acts_old[l], acts_old[l + 1], nullptr, r.batch, w, issued, skipped);
-                BARRIER();
-            }
-            const int blk_lo = r.frontier_skip ? fin_x / B : 0;
-            const int jmax = min(B, T_);
-            for (int j = 0; j < jmax; ++j) {
-                if (j >= 1)
-                    for (int l = 0; l < m.L; ++l) {
-                        jgs_hidden_phase<T>(s, m, r, l, j, B, blk_lo);
-                        BARRIER();
-                    }
-                jgs_output_phase<T>(m, r, j, B, blk_lo);
-                BARRIER();
-                if (m.C > 1) {
-                    jgs_commit_phase<T>(m, r, j, B, blk_lo);
-                    BARRIER();
-                }
-                iterations++;
-            }
-            jgs_copy_or_compare<T>(m, r, true, p);
-            BARRIER();
-            const int any = ld_volatile_i32(&ctl->agg_any[p]);
-            const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
-            book_samples(r, p, k, k == cap, false, true);
-            reset_other_parity(r, p);
-            fin_h = max(fin_h, fin_x);
-            // after outer iteration k the first k blocks are final (proof of Prop. 2)
-            fin_x = any ? max(min(k * B, T_), min(mf + 1, T_)) : T_;
-            if (!any || k == cap) {
-                if (any && cap < M) status = JS_NOT_CONVERGED;
-                break;
-            }
-        }
-        frontier = fin_x;
-        goto done;
-    }
-
-done:
-#undef BARRIER
-    if (threadIdx.x == 0) {
-        atomicAdd(&ctl->tiles_issued, issued);
-        atomicAdd(&ctl->tiles_skipped, skipped);
-        if (blockIdx.x == 0) {
-            ctl->iterations = iterations;
-            ctl->frontier = frontier;
-            ctl->status = alive ? status : JS_ERR_TIMEOUT;
-        }
-    }
+template <typename T>
+__global__ void __launch_bounds__(NTHREADS) made_generic_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ RunArgs r)
+{
+    __shared__ Smem s;
+    GenericEngine<T> e(s, m, r);
+    const DriverResult res = made_driver(e, m, r);
+    driver_finish(r, res, e.issued, e.skipped);
 }
 
 }  // namespace

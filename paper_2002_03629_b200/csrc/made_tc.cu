@@ -1,0 +1,687 @@
+// Tensor-core path of the masked-MLP sampler for sm_100a.
+//
+// One persistent cooperative kernel runs the whole solver.  Every layer of the
+// masked network is a GEMM  D[128 samples x BN units] = A[128 x K] * W[BN x K]^T
+// on the 5th-generation tensor cores: operands arrive in shared memory by TMA
+// (128-byte swizzle, K-major), one elected thread issues tcgen05.mma with the
+// fp32 accumulator in tensor memory, and four epilogue warps read it back with
+// tcgen05.ld.  Masked (all-zero) K blocks beyond a tile's last live input are
+// never loaded; adding exact zeros would not change the fp32 sum, so h_t stays
+// the same function whatever is skipped.  The output layer's epilogue is the
+// sampling step itself (Appendix A.3 of arXiv 2002.03629): bias, fixed noise,
+// threshold or 256-way argmax, compare with the previous iterate, per-sample
+// change flags; logits never reach global memory.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer and TMEM
+// owner, warps 2-5 = epilogue (TMEM lane quadrant = warp index mod 4).
+// All waits are bounded; a wait that gives up raises the abort flag, every role
+// drains, TMEM is freed and the kernel returns JS_ERR_TIMEOUT.
+#include <cuda.h>
+
+#include "js_common.cuh"
+#include "js_model.h"
+#include "made_driver.cuh"
+
+namespace {
+
+constexpr int BM = 128;            // samples per tile (UMMA M)
+constexpr int BK = 64;             // bf16 elements per K block = one 128-byte swizzle row
+constexpr int NTH = 192;
+constexpr int ACC_COLS = 256;      // TMEM columns per accumulator slot (two slots)
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int RING_BYTES = 192 * 1024;
+constexpr int MAX_STAGES = 6;
+constexpr unsigned long long MBAR_WAIT_NS = 2000000000ull;   // 2 s
+
+enum { EPI_HIDDEN = 0, EPI_LOGITS = 1, EPI_BINARY = 2, EPI_CAT = 3 };
+
+// ------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait on an mbarrier phase.  Gives up after MBAR_WAIT_NS or when another
+// thread of the grid has raised the abort flag; then raises the flag itself.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, JsCtl *ctl)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (unsigned i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((i & 63u) == 0u) {
+            if (ld_volatile_i32(&ctl->abort) != 0) break;
+            if (global_ns() - t0 > MBAR_WAIT_NS) break;
+        }
+    }
+    atomicExch(&ctl->abort, 1);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t *dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
+                 "r"(ncols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, 128 x N x 16, bf16 in, fp32 out
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// arrive on an mbarrier once every tcgen05.mma issued so far by this thread has completed
+__device__ __forceinline__ void umma_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's TMEM lane
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory operand descriptor: K-major tile of rows x 64 bf16, 128-byte swizzle,
+// rows 128 bytes apart, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);        // start address
+    d |= (uint64_t)1 << 16;                          // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)(1024 >> 4) << 32;                // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                          // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                          // 128-byte swizzle
+    return d;
+}
+__device__ __forceinline__ uint32_t instr_desc_bf16(int n)
+{
+    // fp32 accumulate, bf16 A and B, both K-major, M = 128
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&h);
+}
+
+struct TcShared {
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2];
+    uint32_t tmem_base;
+};
+
+// ------------------------------------------------------------------ engine
+struct TcEngine {
+    static constexpr bool has_jgs = false;
+    const MadeDev &m;
+    const TcDev &t;
+    const RunArgs &r;
+    TcShared &sh;
+    uint8_t *ring;
+    unsigned epoch = 0;
+    unsigned long long issued = 0, skipped = 0;
+    int warp, lane;
+    // pipeline state, advanced identically by the roles that share it
+    int stage = 0;
+    uint32_t sphase = 0;
+    int acc = 0;
+    uint32_t aphase = 0;
+    bool dead = false;
+    uint32_t tmem_base = 0;
+
+    __device__ TcEngine(const MadeDev &m_, const TcDev &t_, const RunArgs &r_, TcShared &sh_, uint8_t *ring_)
+        : m(m_), t(t_), r(r_), sh(sh_), ring(ring_)
+    {
+        warp = threadIdx.x >> 5;
+        lane = threadIdx.x & 31;
+    }
+
+    __device__ bool barrier()
+    {
+        // epilogue stores of this phase must be visible to the TMA reads of the next one
+        fence_proxy_async();
+        const bool ok = grid_barrier(r.ctl, epoch, r.spin_limit);
+        fence_proxy_async();
+        return ok;
+    }
+
+    __device__ void init(const uint8_t *src)
+    {
+        const size_t n = (size_t)r.batch * m.T;
+        __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+            const uint8_t v = src ? src[i] : (uint8_t)0;
+            if (r.x) r.x[i] = v;
+            a0[i] = __float2bfloat16_rn(m.lut[v]);
+        }
+        if (blockIdx.x == 0) {
+            for (int i = threadIdx.x; i < 2 * r.batch; i += blockDim.x) {
+                r.smp_changed[i] = 0;
+                r.smp_state[i] = 0;
+            }
+            if (threadIdx.x == 0) {
+                r.ctl->agg_any[0] = r.ctl->agg_any[1] = 0;
+                r.ctl->agg_minfirst[0] = r.ctl->agg_minfirst[1] = INT_MAX;
+            }
+        }
+    }
+
+    __device__ uint8_t *stage_a(int s) const { return ring + (size_t)s * t.stage_bytes; }
+    __device__ uint8_t *stage_b(int s) const { return ring + (size_t)s * t.stage_bytes + A_BYTES; }
+    __device__ void advance_stage()
+    {
+        if (++stage == t.n_stages) { stage = 0; sphase ^= 1u; }
+    }
+    __device__ void advance_acc()
+    {
+        acc ^= 1;
+        if (acc == 0) aphase ^= 1u;
+    }
+
+    // live tile range of layer l under the window (tile degrees are monotone)
+    __device__ void live_range(int l, const Win &w, int &nt_lo, int &nt_hi) const
+    {
+        const TcLayer &ly = t.lay[l];
+        const bool is_out = (l == m.L);
+        const int lo_key = is_out ? w.olo + 1 : w.hdeg_lo + 1;   // live iff dmax >= lo_key
+        const int hi_key = is_out ? w.ohi : w.hdeg_hi;           // live iff dmin <= hi_key
+        int a = 0, b = ly.nt;
+        while (a < b) { const int mid = (a + b) >> 1; if (ly.dmax[mid] >= lo_key) b = mid; else a = mid + 1; }
+        nt_lo = a;
+        a = nt_lo; b = ly.nt;
+        while (a < b) { const int mid = (a + b) >> 1; if (ly.dmin[mid] > hi_key) b = mid; else a = mid + 1; }
+        nt_hi = a;
+    }
+
+    __device__ void producer(int l, int nt_lo, int ntiles, int MT)
+    {
+        const TcLayer &ly = t.lay[l];
+        const CUtensorMap *ma = t.tmA + l, *mw = t.tmW + l;
+        const uint32_t bytes = A_BYTES + ly.bn * BK * 2;
+        for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
+            const int nt = nt_lo + id / MT, mt = id % MT;
+            const int kb_end = ly.kb_end[nt];
+            for (int kb = 0; kb < kb_end; ++kb) {
+                if (!mbar_wait(&sh.empty[stage], sphase ^ 1u, r.ctl)) { dead = true; break; }
+                mbar_expect_tx(&sh.full[stage], bytes);
+                tma_load_2d(smem_u32(stage_a(stage)), ma, &sh.full[stage], kb * BK, mt * BM);
+                tma_load_2d(smem_u32(stage_b(stage)), mw, &sh.full[stage], kb * BK, nt * ly.bn);
+                advance_stage();
+            }
+        }
+    }
+
+    __device__ void mma_issuer(int l, int nt_lo, int ntiles, int MT)
+    {
+        const TcLayer &ly = t.lay[l];
+        const uint32_t idesc = instr_desc_bf16(ly.bn);
+        for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
+            const int nt = nt_lo + id / MT;
+            const int kb_end = ly.kb_end[nt];
+            if (!mbar_wait(&sh.tempty[acc], aphase ^ 1u, r.ctl)) { dead = true; break; }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_COLS);
+            for (int kb = 0; kb < kb_end; ++kb) {
+                if (!mbar_wait(&sh.full[stage], sphase, r.ctl)) { dead = true; break; }
+                tc_fence_after();
+                const uint64_t adesc = smem_desc_sw128(smem_u32(stage_a(stage)));
+                const uint64_t bdesc = smem_desc_sw128(smem_u32(stage_b(stage)));
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)       // 16 bf16 = 32 bytes per instruction along K
+                    umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                              (kb > 0 || k > 0) ? 1u : 0u);
+                umma_commit(&sh.empty[stage]);          // frees the stage once these MMAs have read it
+                advance_stage();
+            }
+            if (dead) break;
+            umma_commit(&sh.tfull[acc]);                // accumulator complete
+            advance_acc();
+        }
+    }
+
+    // ---- epilogues: thread = one sample row of the tile, 32 columns at a time
+    __device__ void epi_hidden(int l, int row, int n0, int c0, const float (&v)[32])
+    {
+        const int N = m.n[l + 1];
+        if (row >= r.batch) return;
+        __nv_bfloat16 *out = (__nv_bfloat16 *)m.a[l + 1] + (size_t)row * N;
+        const float *bias = m.bias[l];
+        const int col = n0 + c0;
+        if (col + 32 <= N) {
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+                const float4 b4 = __ldg(reinterpret_cast<const float4 *>(bias + col + i));
+                const float f0 = js_act_fn(m.act, v[i] + b4.x), f1 = js_act_fn(m.act, v[i + 1] + b4.y);
+                const float f2 = js_act_fn(m.act, v[i + 2] + b4.z), f3 = js_act_fn(m.act, v[i + 3] + b4.w);
+                pk[i / 2] = pack_bf16x2(f0, f1);
+                pk[i / 2 + 1] = pack_bf16x2(f2, f3);
+            }
+            uint4 *dst = reinterpret_cast<uint4 *>(out + col);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i)
+                if (col + i < N) out[col + i] = __float2bfloat16_rn(js_act_fn(m.act, v[i] + bias[col + i]));
+        }
+    }
+
+    __device__ void epi_logits(float *zout, int row, int n0, int c0, const float (&v)[32])
+    {
+        const int N = m.n[m.L + 1];
+        if (row >= r.batch) return;
+        const float *bias = m.bias[m.L];
+        const int col = n0 + c0;
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (col + i < N) zout[(size_t)row * N + col + i] = v[i] + bias[col + i];
+    }
+
+    // binary positions d = n0 + c0 + i: threshold against the fixed noise, compare, commit
+    __device__ void epi_binary(const Win &w, int row, int n0, int c0, const float (&v)[32], bool &changed,
+                               int &first)
+    {
+        const int T_ = m.T;
+        if (row >= r.batch) return;
+        const int d0 = n0 + c0;
+        if (d0 >= w.phi || d0 + 32 <= w.plo || d0 >= T_) return;
+        const float *bias = m.bias[m.L];
+        const size_t at = (size_t)row * T_ + d0;
+        __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
+        const float lut0 = m.lut[0], lut1 = m.lut[1];
+        if (d0 + 32 <= T_) {
+            uint32_t xo[8], xn[8];
+            const uint2 *xp = reinterpret_cast<const uint2 *>(r.x + at);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { const uint2 u = xp[i]; xo[2 * i] = u.x; xo[2 * i + 1] = u.y; }
+            uint32_t enc[16];
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+                const float4 b4 = __ldg(reinterpret_cast<const float4 *>(bias + d0 + i));
+                const float4 n4 = __ldg(reinterpret_cast<const float4 *>(r.noise + at + i));
+                const float bb[4] = {b4.x, b4.y, b4.z, b4.w}, nn[4] = {n4.x, n4.y, n4.z, n4.w};
+                uint32_t word = 0;
+                float e[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int d = d0 + i + j;
+                    const uint32_t old = (xo[i / 4] >> (8 * j)) & 0xffu;
+                    uint32_t nv = (uint32_t)js_sample_binary(r.nk, v[i + j] + bb[j], nn[j]);
+                    if (d < w.plo || d >= w.phi) nv = old;
+                    if (nv != old) {
+                        if (!changed) first = d;
+                        changed = true;
+                    }
+                    word |= nv << (8 * j);
+                    e[j] = nv ? lut1 : lut0;
+                }
+                xn[i / 4] = word;
+                enc[i / 2] = pack_bf16x2(e[0], e[1]);
+                enc[i / 2 + 1] = pack_bf16x2(e[2], e[3]);
+            }
+            uint2 *xq = reinterpret_cast<uint2 *>(r.x + at);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) xq[i] = make_uint2(xn[2 * i], xn[2 * i + 1]);
+            uint4 *aq = reinterpret_cast<uint4 *>(a0 + at);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) aq[i] = make_uint4(enc[4 * i], enc[4 * i + 1], enc[4 * i + 2], enc[4 * i + 3]);
+        } else {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int d = d0 + i;
+                if (d >= T_ || d < w.plo || d >= w.phi) continue;
+                const int old = r.x[at + i];
+                const int nv = js_sample_binary(r.nk, v[i] + bias[d], r.noise[at + i]);
+                if (nv != old) {
+                    if (!changed) first = d;
+                    changed = true;
+                    r.x[at + i] = (uint8_t)nv;
+                    a0[at + i] = __float2bfloat16_rn(nv ? lut1 : lut0);
+                }
+            }
+        }
+    }
+
+    // one 256-way position per tile: running argmax of logit + Gumbel noise, lowest index wins ties
+    __device__ void epi_cat_chunk(int row, int d, int c0, const float (&v)[32], float &best, int &bi)
+    {
+        if (row >= r.batch) return;
+        const float *bias = m.bias[m.L] + (size_t)d * 256 + c0;
+        const float *gg = r.noise + ((size_t)row * m.T + d) * 256 + c0;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            const float4 b4 = __ldg(reinterpret_cast<const float4 *>(bias + i));
+            const float4 g4 = __ldg(reinterpret_cast<const float4 *>(gg + i));
+            const float s0 = (v[i] + b4.x) + g4.x, s1 = (v[i + 1] + b4.y) + g4.y;
+            const float s2 = (v[i + 2] + b4.z) + g4.z, s3 = (v[i + 3] + b4.w) + g4.w;
+            if (s0 > best) { best = s0; bi = c0 + i; }
+            if (s1 > best) { best = s1; bi = c0 + i + 1; }
+            if (s2 > best) { best = s2; bi = c0 + i + 2; }
+            if (s3 > best) { best = s3; bi = c0 + i + 3; }
+        }
+    }
+
+    __device__ void epilogue(int l, int kind, const Win &w, bool flag, int parity, float *zout, int nt_lo,
+                             int ntiles, int MT)
+    {
+        const TcLayer &ly = t.lay[l];
+        const int q = warp & 3;
+        bool any_changed = false;
+        int first = INT_MAX;
+        for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
+            const int nt = nt_lo + id / MT, mt = id % MT;
+            if (!mbar_wait(&sh.tfull[acc], aphase, r.ctl)) { dead = true; break; }
+            tc_fence_after();
+            const int row = mt * BM + q * 32 + lane;
+            const int n0 = nt * ly.bn;
+            const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS);
+            float best = -INFINITY;
+            int bi = 0;
+            bool ch = false;
+            int fc = INT_MAX;
+            for (int c0 = 0; c0 < ly.bn; c0 += 32) {
+                float v[32];
+                tmem_ld32(tbase + (uint32_t)c0, v);
+                if (kind == EPI_HIDDEN) epi_hidden(l, row, n0, c0, v);
+                else if (kind == EPI_LOGITS) epi_logits(zout, row, n0, c0, v);
+                else if (kind == EPI_BINARY) epi_binary(w, row, n0, c0, v, ch, fc);
+                else epi_cat_chunk(row, nt, c0, v, best, bi);
+            }
+            if (kind == EPI_CAT && row < r.batch && nt >= w.plo && nt < w.phi) {
+                const size_t at = (size_t)row * m.T + nt;
+                if ((int)r.x[at] != bi) {
+                    r.x[at] = (uint8_t)bi;
+                    ((__nv_bfloat16 *)m.a[0])[at] = __float2bfloat16_rn(m.lut[bi]);
+                    ch = true;
+                    fc = nt;
+                }
+            }
+            if (flag && ch) {
+                r.smp_changed[parity * r.batch + row] = 1;
+                any_changed = true;
+                first = min(first, fc);
+            }
+            // release the accumulator slot
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.tempty[acc]);
+            advance_acc();
+        }
+        if (flag) {
+            const bool wany = __any_sync(0xffffffffu, any_changed);
+            if (wany) {
+                const int wmin = __reduce_min_sync(0xffffffffu, first);
+                if (lane == 0) {
+                    atomicMin(&r.ctl->agg_minfirst[parity], wmin);
+                    atomicOr(&r.ctl->agg_any[parity], 1);
+                }
+            }
+        }
+    }
+
+    // one layer over the window; returns false when there was nothing to do (no barrier needed)
+    __device__ bool gemm_phase(int l, int kind, const Win &w, bool flag, int parity, float *zout)
+    {
+        int nt_lo, nt_hi;
+        live_range(l, w, nt_lo, nt_hi);
+        const int MT = (r.batch + BM - 1) / BM;
+        const int nlive = max(0, nt_hi - nt_lo);
+        const int ntiles = nlive * MT;
+        if (threadIdx.x == 0) {
+            int mine = 0;
+            for (int id = blockIdx.x; id < ntiles; id += gridDim.x) mine++;
+            issued += mine;
+            if (blockIdx.x == 0) skipped += (unsigned long long)(t.lay[l].nt - nlive) * MT;
+        }
+        if (ntiles == 0) return false;
+        if (warp == 0) {
+            if (lane == 0) producer(l, nt_lo, ntiles, MT);
+        } else if (warp == 1) {
+            if (lane == 0) mma_issuer(l, nt_lo, ntiles, MT);
+        } else {
+            epilogue(l, kind, w, flag, parity, zout, nt_lo, ntiles, MT);
+        }
+        return true;
+    }
+
+    __device__ bool forward_logits(float *zout)
+    {
+        const Win w = make_win(0, m.T, 0, m.T);
+        for (int l = 0; l < m.L; ++l) {
+            gemm_phase(l, EPI_HIDDEN, w, false, 0, nullptr);
+            if (!barrier()) return false;
+        }
+        gemm_phase(m.L, EPI_LOGITS, w, false, 0, zout);
+        return barrier();
+    }
+
+    __device__ bool step(const Win &w, bool flag, int parity)
+    {
+        for (int l = 0; l < m.L; ++l)
+            if (gemm_phase(l, EPI_HIDDEN, w, false, 0, nullptr))
+                if (!barrier()) return false;
+        gemm_phase(m.L, m.C == 1 ? EPI_BINARY : EPI_CAT, w, flag, parity, nullptr);
+        return barrier();
+    }
+};
+
+__global__ void __launch_bounds__(NTH, 1)
+made_tc_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ TcDev t, const __grid_constant__ RunArgs r)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ TcShared sh;
+    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+    }
+    if (warp == 1) tmem_alloc(&sh.tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    TcEngine e(m, t, r, sh, ring);
+    e.tmem_base = sh.tmem_base;
+    DriverResult res = made_driver(e, m, r);
+    if (e.dead) res.alive = false;
+
+    // leave: let copies still in flight land (only possible after an aborted wait), free TMEM
+    tc_fence_before();
+    __syncthreads();
+    if (!res.alive || ld_volatile_i32(&r.ctl->abort) != 0) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+        res.alive = false;
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(e.tmem_base, 512);
+    }
+    driver_finish(r, res, e.issued, e.skipped);
+}
+
+}  // namespace
+
+// --------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+        return nullptr;
+    fn = (EncodeTiledFn)p;
+    return fn;
+}
+
+// 2-D bf16 row-major tensor [rows][cols], box = 64 columns x box_rows rows, 128-byte swizzle
+static bool encode_map(CUtensorMap *out, const void *base, int rows, int cols, int box_rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Builds the tensor-core view of a model.  Returns 1 if the model qualifies, 0 if it
+// does not (the CUDA-core path then serves it), negative on CUDA errors.
+int js_tc_prepare(js_model *mo)
+{
+    const MadeDev &v = mo->made;
+    TcDev &t = mo->tc;
+    mo->tc_ok = 0;
+    if (v.prec != JS_BF16) return 0;
+    if (!(v.C == 1 || v.C == 256)) return 0;
+    for (int l = 0; l <= v.L; ++l)
+        if (v.n[l] % 8 != 0) return 0;
+    if (!get_encode_fn()) return 0;
+    const int L = v.L;
+    bool wide = (v.C == 256);
+    t.stage_bytes = A_BYTES + (wide ? 256 : 128) * BK * 2;
+    t.n_stages = RING_BYTES / t.stage_bytes;
+    if (t.n_stages > MAX_STAGES) t.n_stages = MAX_STAGES;
+    std::vector<CUtensorMap> mapsA(L + 1), mapsW(L + 1);
+    for (int l = 0; l <= L; ++l) {
+        const int bn = (l == L && wide) ? 256 : 128;
+        const int N = v.n[l + 1], K = v.n[l], nt = (N + bn - 1) / bn;
+        std::vector<int> kb(nt), dmin(nt), dmax(nt);
+        const std::vector<int> &dout = mo->host_deg[l + 1], &din = mo->host_deg[l];
+        for (int i = 0; i < nt; ++i) {
+            int lo = INT32_MAX, hi = 0;
+            for (int u = i * bn; u < std::min(N, (i + 1) * bn); ++u) { lo = std::min(lo, dout[u]); hi = std::max(hi, dout[u]); }
+            int ke = K;
+            while (ke > 0 && !(l == L ? din[ke - 1] < hi : din[ke - 1] <= hi)) --ke;
+            kb[i] = std::max(1, (ke + BK - 1) / BK);
+            dmin[i] = lo; dmax[i] = hi;
+            if (i > 0 && (dmin[i] < dmin[i - 1] || dmax[i] < dmax[i - 1])) return 0;   // needs sorted degrees
+        }
+        void *p = nullptr;
+        for (std::vector<int> *src : {&kb, &dmin, &dmax}) {
+            if (cudaMalloc(&p, nt * sizeof(int)) != cudaSuccess) return JS_ERR_CUDA;
+            mo->allocs.push_back(p);
+            if (cudaMemcpy(p, src->data(), nt * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return JS_ERR_CUDA;
+            if (src == &kb) t.lay[l].kb_end = (const int *)p;
+            else if (src == &dmin) t.lay[l].dmin = (const int *)p;
+            else t.lay[l].dmax = (const int *)p;
+        }
+        t.lay[l].bn = bn;
+        t.lay[l].nt = nt;
+        if (!encode_map(&mapsA[l], v.a[l], mo->rows, K, BM)) return 0;
+        if (!encode_map(&mapsW[l], v.W[l], N, K, bn)) return 0;
+    }
+    void *pa = nullptr, *pw = nullptr;
+    if (cudaMalloc(&pa, (L + 1) * sizeof(CUtensorMap)) != cudaSuccess) return JS_ERR_CUDA;
+    mo->allocs.push_back(pa);
+    if (cudaMalloc(&pw, (L + 1) * sizeof(CUtensorMap)) != cudaSuccess) return JS_ERR_CUDA;
+    mo->allocs.push_back(pw);
+    if (cudaMemcpy(pa, mapsA.data(), (L + 1) * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess) return JS_ERR_CUDA;
+    if (cudaMemcpy(pw, mapsW.data(), (L + 1) * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess) return JS_ERR_CUDA;
+    t.tmA = (const CUtensorMap *)pa;
+    t.tmW = (const CUtensorMap *)pw;
+
+    const int smem = RING_BYTES + 1024;
+    if (cudaFuncSetAttribute(made_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return 0;
+    int dev = 0, sms = 0, per_sm = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, made_tc_kernel, NTH, smem) != cudaSuccess || per_sm < 1)
+        return 0;
+    mo->tc_max_grid = sms;      // one CTA per SM: each owns all 512 TMEM columns
+    mo->tc_ok = 1;
+    return 1;
+}
+
+int js_launch_made_tc(const js_model *mo, const RunArgs &r, cudaStream_t stream)
+{
+    const MadeDev &v = mo->made;
+    const TcDev &t = mo->tc;
+    const int MT = (r.batch + BM - 1) / BM;
+    int tiles = 1;
+    for (int l = 0; l <= v.L; ++l) tiles = std::max(tiles, t.lay[l].nt * MT);
+    const int grid = std::max(1, std::min(mo->tc_max_grid, tiles));
+    void *args[3] = {(void *)&v, (void *)&t, (void *)&r};
+    cudaError_t e = cudaLaunchCooperativeKernel((const void *)made_tc_kernel, dim3(grid), dim3(NTH), args,
+                                                RING_BYTES + 1024, stream);
+    return e == cudaSuccess ? 0 : (int)e;
+}

@@ -82,18 +82,37 @@ CAT = si.scaled(si.CONFIGS["made_cat"], D=24, H=(128, 96), batch=9)
 CHAIN = si.scaled(si.CONFIGS["made_4096"], D=256, H=(256, 256, 256, 256), batch=130, w_var_scale=4.0)
 
 CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN}
+# kernel path: 1 = CUDA-core kernels, 0 = tensor-core kernels (bf16 models only)
+COMBOS = [(n, 1) for n in CASES] + [(n, 0) for n in CASES if n != "tiny"]
+COMBO_IDS = [f"{n}-{'tc' if p == 0 else 'cc'}" for n, p in COMBOS]
 _cache = {}
+_path = {"v": 1}
 
 
-def case(name, path=1):
+def case(name, path=None):
+    path = _path["v"] if path is None else path
     key = (name, path)
     if key not in _cache:
         _cache[key] = Case(CASES[name], path=path)
     return _cache[key]
 
 
+@pytest.fixture(params=[1, 0], ids=["cc", "tc"], autouse=True)
+def kernel_path(request):
+    """Every test runs once per kernel path; fp32-only cases skip the tensor-core pass."""
+    _path["v"] = request.param
+    yield request.param
+    _path["v"] = 1
+
+
+def _skip_if_not_applicable(name):
+    if _path["v"] == 0 and CASES[name].prec != si.PREC_BF16:
+        pytest.skip("tensor-core kernels serve bf16 models only")
+
+
 @pytest.mark.parametrize("name", list(CASES))
 def test_logits_match_oracle(name):
+    _skip_if_not_applicable(name)
     c = case(name)
     cfg, p = c.cfg, c.p
     x = si.random_init(cfg, salt=5)
@@ -110,10 +129,12 @@ def test_logits_match_oracle(name):
 @pytest.mark.parametrize("name", list(CASES))
 @pytest.mark.parametrize("skip", [1, 0])
 def test_jacobi_matches_sequential_and_counts(name, skip):
+    _skip_if_not_applicable(name)
     c = case(name)
     c.model.set_option(c.p.JS_OPT_FRONTIER_SKIP, skip)
     try:
         c.check(c.p.JS_JACOBI)
+        assert c.model.stats().path == _path["v"]          # the requested kernels really ran
         c.check(c.p.JS_JACOBI, init=si.random_init(c.cfg, salt=1))
     finally:
         c.model.set_option(c.p.JS_OPT_FRONTIER_SKIP, 1)
@@ -122,6 +143,7 @@ def test_jacobi_matches_sequential_and_counts(name, skip):
 @pytest.mark.parametrize("name", list(CASES))
 @pytest.mark.parametrize("seq_skip", [0, 1])
 def test_sequential_and_gauss_seidel(name, seq_skip):
+    _skip_if_not_applicable(name)
     c = case(name)
     p, cfg = c.p, c.cfg
     c.model.set_option(p.JS_OPT_SEQ_SKIP, seq_skip)
@@ -140,6 +162,7 @@ def test_sequential_and_gauss_seidel(name, seq_skip):
                                          ("chain", (32, 64))])
 @pytest.mark.parametrize("skip", [1, 0])
 def test_hybrids(name, blocks, skip):
+    _skip_if_not_applicable(name)
     c = case(name)
     p = c.p
     c.model.set_option(p.JS_OPT_FRONTIER_SKIP, skip)
@@ -154,6 +177,7 @@ def test_hybrids(name, blocks, skip):
 
 @pytest.mark.parametrize("name", ["bin", "chain"])
 def test_max_iters_returns_last_iterate(name):
+    _skip_if_not_applicable(name)
     c = case(name)
     p = c.p
     _, it_full = c.oracle_counts(p.JS_JACOBI)
