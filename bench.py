@@ -222,6 +222,12 @@ def run_ours(args, cfg):
     barrier()
     ms = [s.elapsed_time(e) for s, e in ev]
     total_ms = float(sum(ms))
+    if sampler:
+        # the timed region is milliseconds long: keep the same load running (untimed) until
+        # nvidia-smi has had time to take a few samples of the clocks under it
+        t_end = time.perf_counter() + 0.8
+        while time.perf_counter() < t_end:
+            step()
     clocks = sampler.stop() if sampler else None
 
     # ---- end to end: pinned host noise in, samples out, inside the timed region
