@@ -27,6 +27,7 @@
 #ifndef JACOBI_SAMPLE_H
 #define JACOBI_SAMPLE_H
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -151,6 +152,46 @@ int js_get_stats(const js_model *m, js_stats *out);
 
 const char *js_strerror(int code);
 const char *js_last_cuda_error(void);   /* text of the last failed CUDA call on this thread */
+
+/*
+ * jacobi_sample_noalloc - JS_JACOBI sampling of a small fp32 masked MLP without any
+ * device-memory allocation.  The paper has no counterpart for this entry point; it exists
+ * for callers that are not allowed to call cudaMalloc when they sample (a real-time loop
+ * that must not block on the allocator, a process whose device memory belongs to another
+ * framework's pool), and who therefore cannot use js_made_create.
+ *
+ * The caller owns and passes everything: the UNMASKED fp32 weights W_dev[l] [n[l+1]][n[l]],
+ * biases b_dev[l] and the input table lut_dev as DEVICE pointers (masks of the default
+ * degree rule are applied on the fly; there are no custom degrees), the noise, the optional
+ * start iterate and the outputs, with the layouts of jacobi_sample.  All other memory the
+ * kernel needs is one fixed device array inside the library, js_noalloc_scratch_limit()
+ * bytes (4 MiB), which every GPU that loads the library holds until the process exits.
+ * A shape whose scratch (js_noalloc_scratch_needed) exceeds it is rejected with JS_ERR_ARG
+ * and a message in js_noalloc_last_error().  The call makes no cudaMalloc/cudaFree and calls
+ * no allocating library routine.
+ *
+ * All calls share the one array and find the previous call's contents in it; the kernel
+ * clears what must start at zero.  Calls that overlap on the GPU race on it: serialise them.
+ * The first call on each device looks up the array's device address (with that device
+ * current), so make it before any stream capture begins.  Runs on one CTA: meant for small
+ * models.  Results equal jacobi_sample(..., JS_JACOBI, ...) on the same fp32 model: same
+ * samples, same out_iters, same return codes (0, JS_NOT_CONVERGED, negative on error).
+ */
+typedef struct {
+    int T, C, L;
+    int H[8];
+    int act;                    /* js_act */
+    const float *W_dev[9];      /* device pointers, l = 0..L */
+    const float *b_dev[9];
+    const float *lut_dev;       /* device pointer, 2 entries (binary) or C entries */
+} js_noalloc_made;
+
+int jacobi_sample_noalloc(const js_noalloc_made *net, int batch, const float *noise_dev, int nk,
+                          const uint8_t *init_dev, int max_iters, uint8_t *out_samples_dev,
+                          int32_t *out_iters_dev, void *cuda_stream);
+size_t js_noalloc_scratch_limit(void);
+size_t js_noalloc_scratch_needed(const js_noalloc_made *net, int batch);
+const char *js_noalloc_last_error(void);
 
 #ifdef __cplusplus
 }

@@ -42,6 +42,11 @@ class _ConvDesc(C.Structure):
                 ("lut", C.POINTER(C.c_float)), ("n_lut", C.c_int), ("max_batch", C.c_int)]
 
 
+class _NoallocMade(C.Structure):
+    _fields_ = [("T", C.c_int), ("C", C.c_int), ("L", C.c_int), ("H", C.c_int * 8), ("act", C.c_int),
+                ("W_dev", C.c_void_p * 9), ("b_dev", C.c_void_p * 9), ("lut_dev", C.c_void_p)]
+
+
 class JsStats(C.Structure):
     _fields_ = [("iterations", C.c_int), ("batch_iters_max", C.c_int), ("final_frontier", C.c_int),
                 ("tiles_issued", C.c_longlong), ("tiles_skipped", C.c_longlong), ("path", C.c_int),
@@ -70,6 +75,11 @@ def load_library():
     lib.js_strerror.argtypes = [ip]
     lib.js_strerror.restype = C.c_char_p
     lib.js_last_cuda_error.restype = C.c_char_p
+    lib.jacobi_sample_noalloc.argtypes = [C.POINTER(_NoallocMade), ip, vp, ip, vp, ip, vp, vp, vp]
+    lib.js_noalloc_scratch_limit.restype = C.c_size_t
+    lib.js_noalloc_scratch_needed.argtypes = [C.POINTER(_NoallocMade), ip]
+    lib.js_noalloc_scratch_needed.restype = C.c_size_t
+    lib.js_noalloc_last_error.restype = C.c_char_p
     _lib = lib
     return lib
 
@@ -207,3 +217,47 @@ def js_forward_logits(model: Model, x: torch.Tensor, logits: torch.Tensor, strea
     rc = load_library().js_forward_logits(model._h, batch, _dev(x, torch.uint8, "x"),
                                           _dev(logits, torch.float32, "logits"), _stream_ptr(stream))
     return _check(rc, "js_forward_logits")
+
+
+def _noalloc_net(T: int, Cc: int, H: Sequence[int], act: int, W: List[torch.Tensor], b: List[torch.Tensor],
+                 lut: torch.Tensor) -> _NoallocMade:
+    net = _NoallocMade()
+    net.T, net.C, net.L, net.act = T, Cc, len(H), act
+    for i, h in enumerate(H):
+        net.H[i] = h
+    for l in range(len(H) + 1):
+        net.W_dev[l] = _dev(W[l], torch.float32, f"W[{l}]").value
+        net.b_dev[l] = _dev(b[l], torch.float32, f"b[{l}]").value
+    net.lut_dev = _dev(lut, torch.float32, "lut").value
+    return net
+
+
+def jacobi_sample_noalloc(T: int, Cc: int, H: Sequence[int], act: int, W: List[torch.Tensor],
+                          b: List[torch.Tensor], lut: torch.Tensor, noise: torch.Tensor, nk: int,
+                          init: Optional[torch.Tensor], max_iters: int, out_samples: torch.Tensor,
+                          out_iters: Optional[torch.Tensor] = None, stream=None) -> int:
+    """jacobi_sample_noalloc of the C ABI: for callers that may not allocate device memory.  Every
+    tensor (unmasked fp32 weights included) is a CUDA tensor the caller already owns; the library
+    allocates nothing and uses its built-in scratch array.  Calls must not overlap on the GPU."""
+    lib = load_library()
+    net = _noalloc_net(T, Cc, H, act, W, b, lut)
+    rc = lib.jacobi_sample_noalloc(C.byref(net), out_samples.shape[0], _dev(noise, torch.float32, "noise"), nk,
+                                   _dev(init, torch.uint8, "init"), max_iters,
+                                   _dev(out_samples, torch.uint8, "out_samples"),
+                                   _dev(out_iters, torch.int32, "out_iters"), _stream_ptr(stream))
+    if rc < 0:
+        raise JsError(rc, "jacobi_sample_noalloc: " + (lib.js_noalloc_last_error().decode()
+                                                       or lib.js_strerror(rc).decode()))
+    return rc
+
+
+def noalloc_scratch_needed(T: int, Cc: int, H: Sequence[int], batch: int) -> int:
+    net = _NoallocMade()
+    net.T, net.C, net.L = T, Cc, len(H)
+    for i, h in enumerate(H):
+        net.H[i] = h
+    return int(load_library().js_noalloc_scratch_needed(C.byref(net), batch))
+
+
+def noalloc_scratch_limit() -> int:
+    return int(load_library().js_noalloc_scratch_limit())
