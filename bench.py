@@ -222,7 +222,7 @@ def run_ours(args, cfg):
     barrier()
     ms = [s.elapsed_time(e) for s, e in ev]
     total_ms = float(sum(ms))
-    if sampler:
+    if sampler and not args.profile:
         # the timed region is milliseconds long: keep the same load running (untimed) until
         # nvidia-smi has had time to take a few samples of the clocks under it
         t_end = time.perf_counter() + 0.8
@@ -233,7 +233,7 @@ def run_ours(args, cfg):
     # ---- end to end: pinned host noise in, samples out, inside the timed region
     barrier()
     t_e2e = []
-    for _ in range(args.steps):
+    for _ in range(1 if args.profile else args.steps):
         flush.zero_()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
@@ -242,11 +242,11 @@ def run_ours(args, cfg):
         h_out.copy_(out, non_blocking=True)
         torch.cuda.synchronize()
         t_e2e.append(time.perf_counter() - t0)
-    e2e_s = float(sum(t_e2e))
+    e2e_s = float(sum(t_e2e)) * (args.steps / len(t_e2e))
 
     # ---- the same kernels in strict sequential order (speedup denominators)
     seq = {}
-    if args.seq and rank == 0:
+    if args.seq and rank == 0 and not args.profile:
         for name, opt in (("seq_skip", 1), ("seq_full", 0)):
             if name == "seq_full" and args.seq == "skip":
                 continue
@@ -309,7 +309,7 @@ def run_ours(args, cfg):
                 line["speedup_vs_" + k[:-3]] = seq[k] / ms_launch
 
     # ---- CPU baseline: the oracle on a bounded sample of the same workload
-    if not args.no_cpu_baseline:
+    if not args.no_cpu_baseline and not args.profile:
         import oracle
         oracle.build()
         W, b, lut, noise2 = make_inputs(cfg)
@@ -341,6 +341,8 @@ def main():
     ap.add_argument("--ref-samples", type=int, default=0,
                     help="samples per step of the CPU oracle (0: sized for roughly 15 s of CPU work)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--profile", action="store_true",
+                    help="only the warm-up and the timed steps (for short runs under a profiler)")
     args = ap.parse_args()
     cfg = si.CONFIGS[args.workload]
     if args.batch:

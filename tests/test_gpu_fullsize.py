@@ -1,0 +1,104 @@
+"""Parity at the benchmark's full sizes, in the launch configuration bench.py times
+(tensor-core kernels, zero start, Jacobi), plus the hybrids the workloads name.
+
+Samples are checked against the oracle's feedforward pass for EVERY sample of the
+batch (all solvers must return exactly that, Propositions 1-2); iteration counts and
+logits are checked on a few samples, which the oracle can afford one by one."""
+import time
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from parity import check_samples, logits_close
+
+pytestmark = pytest.mark.gpu
+_cases = {}
+
+
+def full_case(name):
+    if name in _cases:
+        return _cases[name]
+    import __graft_entry__ as ge
+    ge.build()
+    import paper_2002_03629_b200 as p
+    cfg = si.CONFIGS[name]
+    W, b = si.made_weights(cfg)
+    lut = si.made_lut(cfg)
+    noise = si.draw_noise(cfg)
+    orc = oracle.from_config(cfg, W, b, lut)
+    model = p.Model.from_config(cfg, W, b, lut)
+    del W, b
+    xstar = orc.sequential_batch(noise, cfg.noise_kind, threads=16)
+    _cases.clear()                      # one full-size model at a time on the host
+    _cases[name] = (p, cfg, orc, model, noise, torch.from_numpy(noise).cuda(), xstar)
+    return _cases[name]
+
+
+def run(p, cfg, model, d_noise, mode, block=0):
+    out = torch.full((cfg.batch, cfg.D), 255, dtype=torch.uint8, device="cuda")
+    iters = torch.full((cfg.batch,), -1, dtype=torch.int32, device="cuda")
+    rc = p.jacobi_sample(model, d_noise, cfg.noise_kind, None, mode, block, 0, out, iters)
+    assert rc == 0
+    return out.cpu().numpy(), iters.cpu().numpy()
+
+
+@pytest.mark.parametrize("name", ["made_784", "made_4096", "made_cat"])
+def test_full_size_jacobi_and_hybrids(name):
+    p, cfg, orc, model, noise, d_noise, xstar = full_case(name)
+    nk = cfg.noise_kind
+    # Jacobi, as benchmarked
+    x, it = run(p, cfg, model, d_noise, p.JS_JACOBI)
+    assert model.stats().path == 0, "the tensor-core kernels must serve the benchmark workloads"
+    audit = check_samples(orc, x, xstar, noise, nk)
+    print(f"{name}: jacobi iters mean {it.mean():.3f} max {it.max()} excused {audit}")
+    n = 12 if name != "made_cat" else 6
+    ref = orc.map_batch(lambda i: orc.jacobi(noise[i], nk)[1], n, threads=16)
+    clean = [i for i in range(n) if i not in audit["excused_samples"]]
+    np.testing.assert_array_equal(it[clean], np.array(ref)[clean])
+    assert 1 <= it.min() and it.max() <= cfg.D
+    # sequential order with the same kernels (banded)
+    model.set_option(p.JS_OPT_SEQ_SKIP, 1)
+    seq = torch.empty((cfg.batch, cfg.D), dtype=torch.uint8, device="cuda")
+    assert p.sequential_sample(model, d_noise, nk, seq) == 0
+    model.set_option(p.JS_OPT_SEQ_SKIP, 0)
+    check_samples(orc, seq.cpu().numpy(), xstar, noise, nk)
+    # GS-Jacobi with the block sizes the workload names
+    for B in cfg.blocks:
+        x, it = run(p, cfg, model, d_noise, p.JS_GS_JACOBI, B)
+        audit = check_samples(orc, x, xstar, noise, nk)
+        ref = orc.map_batch(lambda i: orc.gs_jacobi(noise[i], nk, B)[1], 4, threads=16)
+        clean = [i for i in range(4) if i not in audit["excused_samples"]]
+        np.testing.assert_array_equal(it[clean], np.array(ref)[clean])
+        assert it.min() >= -(-cfg.D // B) and it.max() <= cfg.D
+
+
+@pytest.mark.parametrize("name", ["made_4096", "made_cat"])
+def test_full_size_jacobi_gs(name):
+    p, cfg, orc, model, noise, d_noise, xstar = full_case(name)
+    nk = cfg.noise_kind
+    B = cfg.blocks[0]
+    t0 = time.perf_counter()
+    x, it = run(p, cfg, model, d_noise, p.JS_JACOBI_GS, B)
+    print(f"{name}: jacobi-gs B={B} took {time.perf_counter() - t0:.2f} s, outer iters max {it.max()}")
+    audit = check_samples(orc, x, xstar, noise, nk)
+    ref = orc.map_batch(lambda i: orc.jacobi_gs(noise[i], nk, B)[1], 2, threads=2)
+    clean = [i for i in range(2) if i not in audit["excused_samples"]]
+    np.testing.assert_array_equal(it[clean], np.array(ref)[clean])
+    assert it.max() <= -(-cfg.D // B)
+
+
+@pytest.mark.parametrize("name", ["made_784", "made_4096", "made_cat"])
+def test_full_size_logits_on_sampled_rows(name):
+    p, cfg, orc, model, noise, d_noise, xstar = full_case(name)
+    x = si.random_init(cfg, salt=9)
+    logits = torch.empty((cfg.batch, cfg.D, cfg.C), dtype=torch.float32, device="cuda")
+    assert p.js_forward_logits(model, torch.from_numpy(x).cuda(), logits) == 0
+    rows = [0, cfg.batch // 2, cfg.batch - 1]
+    got = logits[rows].cpu().numpy()
+    ref = np.stack(orc.map_batch(lambda i: orc.forward_logits(x[rows[i]]), len(rows), threads=3))
+    err, ok = logits_close(got, ref, 2e-2)
+    print(f"{name}: max relative logit error {err:.3e}")
+    assert ok, err
