@@ -134,7 +134,8 @@ typedef enum {
     JS_OPT_SEQ_SKIP = 1,       /* 0 (default): sequential_sample recomputes everything each step; 1: only the band that changed */
     JS_OPT_SPIN_LIMIT = 2,     /* polls before a device-side wait gives up (default 1<<22) */
     JS_OPT_PATH = 3,           /* 0 (default): tensor-core kernels where the model allows; 1: CUDA-core kernels only */
-    JS_OPT_COMPACT = 4         /* 1 (default): move finished samples out of the working batch */
+    JS_OPT_COMPACT = 4,        /* 1 (default): move finished samples out of the working batch */
+    JS_OPT_TRACE = 5           /* 0 (default); 1: record device timestamps of the next calls (js_get_trace) */
 } js_option;
 int js_set_option(js_model *m, int option, int value);
 
@@ -149,6 +150,13 @@ typedef struct {
     int status;                /* the call's return value */
 } js_stats;
 int js_get_stats(const js_model *m, js_stats *out);
+
+/* Device-side timeline of the most recent call made with JS_OPT_TRACE on (tensor-core kernels):
+ * globaltimer nanoseconds, layout [2][256][8] = [first CTA, last CTA][phase][slot]; a phase is one
+ * layer of one forward pass; slots: 0 phase start, 1 first operands landed, 2 last MMA issued,
+ * 3 accumulator complete, 4 epilogue stored, 5 left the grid barrier; 0 = not recorded.
+ * Copies at most `capacity` values to the HOST array `out`, returns how many. */
+int js_get_trace(const js_model *m, unsigned long long *out, int capacity);
 
 const char *js_strerror(int code);
 const char *js_last_cuda_error(void);   /* text of the last failed CUDA call on this thread */

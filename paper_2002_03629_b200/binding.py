@@ -15,7 +15,7 @@ JS_ACT_RELU, JS_ACT_GELU_TANH = 0, 1
 JS_F32, JS_BF16 = 0, 1
 JS_OK, JS_NOT_CONVERGED = 0, 1
 JS_ERR_ARG, JS_ERR_UNSUPPORTED, JS_ERR_CUDA, JS_ERR_TIMEOUT = -1, -2, -3, -4
-JS_OPT_FRONTIER_SKIP, JS_OPT_SEQ_SKIP, JS_OPT_SPIN_LIMIT, JS_OPT_PATH, JS_OPT_COMPACT = 0, 1, 2, 3, 4
+JS_OPT_FRONTIER_SKIP, JS_OPT_SEQ_SKIP, JS_OPT_SPIN_LIMIT, JS_OPT_PATH, JS_OPT_COMPACT, JS_OPT_TRACE = 0, 1, 2, 3, 4, 5
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libjacobi_sample.so")
 _lib = None
@@ -72,6 +72,7 @@ def load_library():
     lib.js_forward_logits.argtypes = [vp, ip, vp, vp, vp]
     lib.js_set_option.argtypes = [vp, ip, ip]
     lib.js_get_stats.argtypes = [vp, C.POINTER(JsStats)]
+    lib.js_get_trace.argtypes = [vp, vp, ip]
     lib.js_strerror.argtypes = [ip]
     lib.js_strerror.restype = C.c_char_p
     lib.js_last_cuda_error.restype = C.c_char_p
@@ -180,6 +181,12 @@ class Model:
         s = JsStats()
         _check(load_library().js_get_stats(self._h, C.byref(s)), "js_get_stats")
         return s
+
+    def trace(self) -> np.ndarray:
+        """js_get_trace: device timestamps [2 CTAs][256 phases][8 slots] of the last traced call."""
+        buf = np.zeros((2, 256, 8), dtype=np.uint64)
+        _check(load_library().js_get_trace(self._h, buf.ctypes.data_as(C.c_void_p), buf.size), "js_get_trace")
+        return buf
 
     def close(self) -> None:
         if self._h:

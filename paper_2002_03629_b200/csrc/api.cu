@@ -164,6 +164,7 @@ int common_scratch(js_model *m, int T)
     if ((rc = dev_alloc<int>(m, &m->smp_state, 2 * (size_t)m->rows, true)) != JS_OK) return rc;
     if ((rc = dev_alloc<uint8_t>(m, &m->x_old, (size_t)m->rows * T, true)) != JS_OK) return rc;
     if ((rc = dev_alloc<uint8_t>(m, &m->x_tmp, (size_t)m->rows * T, true)) != JS_OK) return rc;
+    if ((rc = dev_alloc<unsigned long long>(m, &m->trace, 2 * JS_TRACE_PHASES * JS_TRACE_SLOTS, true)) != JS_OK) return rc;
     return JS_OK;
 }
 
@@ -185,6 +186,8 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
     r.frontier_skip = m->opt_frontier_skip;
     r.seq_skip = m->opt_seq_skip;
     r.spin_limit = (unsigned)m->opt_spin_limit;
+    r.trace = m->opt_trace ? m->trace : nullptr;
+    if (r.trace) CU_TRY(cudaMemsetAsync(m->trace, 0, sizeof(unsigned long long) * 2 * JS_TRACE_PHASES * JS_TRACE_SLOTS, st));
     CU_TRY(cudaMemsetAsync(m->ctl, 0, sizeof(JsCtl), st));
 
     int used_path = 1;
@@ -334,8 +337,18 @@ int js_set_option(js_model *m, int option, int value)
     case JS_OPT_SPIN_LIMIT: if (value < 0) return JS_ERR_ARG; m->opt_spin_limit = value; return JS_OK;
     case JS_OPT_PATH: if (value != 0 && value != 1) return JS_ERR_ARG; m->opt_path = value; return JS_OK;
     case JS_OPT_COMPACT: m->opt_compact = value ? 1 : 0; return JS_OK;
+    case JS_OPT_TRACE: m->opt_trace = value ? 1 : 0; return JS_OK;
     default: return JS_ERR_ARG;
     }
+}
+
+int js_get_trace(const js_model *m, unsigned long long *out, int capacity)
+{
+    if (!m || !out || capacity < 0) return JS_ERR_ARG;
+    const int n = 2 * JS_TRACE_PHASES * JS_TRACE_SLOTS;
+    const int k = capacity < n ? capacity : n;
+    if (cudaMemcpy(out, m->trace, sizeof(unsigned long long) * k, cudaMemcpyDeviceToHost) != cudaSuccess) return JS_ERR_CUDA;
+    return k;
 }
 
 int js_get_stats(const js_model *m, js_stats *out)

@@ -9,6 +9,8 @@
 #include "../../include/jacobi_sample.h"
 
 #define JS_MAXL 8
+#define JS_TRACE_PHASES 256
+#define JS_TRACE_SLOTS 8
 #define JS_GT 64          // output-tile edge of the CUDA-core GEMM phases
 
 enum { KM_JACOBI = 0, KM_SEQ = 1, KM_GS_JACOBI = 2, KM_JACOBI_GS = 3, KM_FORWARD = 4 };
@@ -61,6 +63,7 @@ struct RunArgs {
     int frontier_skip, seq_skip;
     unsigned spin_limit;
     JsCtl *ctl;
+    unsigned long long *trace;   // [2 CTAs][JS_TRACE_PHASES][JS_TRACE_SLOTS] globaltimer stamps, or NULL
 };
 
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)

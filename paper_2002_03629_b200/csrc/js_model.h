@@ -19,7 +19,7 @@ struct TcDev {
     const CUtensorMap *tmA;      // [L+1] activations a[l], box 64 x 128
     const CUtensorMap *tmW;      // [L+1] masked weights W[l], box 64 x bn
     TcLayer lay[JS_MAXL + 1];
-    int stage_bytes, n_stages;
+    int stage_bytes, n_stages, smem_bytes;
 };
 
 struct js_model {
@@ -33,7 +33,8 @@ struct js_model {
     JsCtl *ctl = nullptr;
     int *smp_changed = nullptr, *smp_state = nullptr;
     uint8_t *x_old = nullptr, *x_tmp = nullptr;
-    int opt_frontier_skip = 1, opt_seq_skip = 0, opt_spin_limit = 1 << 22, opt_path = 0, opt_compact = 1;
+    unsigned long long *trace = nullptr;
+    int opt_frontier_skip = 1, opt_seq_skip = 0, opt_spin_limit = 1 << 22, opt_path = 0, opt_compact = 1, opt_trace = 0;
     int max_grid_generic = 0;
     TcDev tc{};
     int tc_ok = 0, tc_max_grid = 0;

@@ -29,8 +29,10 @@ constexpr int BK = 64;             // bf16 elements per K block = one 128-byte s
 constexpr int NTH = 192;
 constexpr int ACC_COLS = 256;      // TMEM columns per accumulator slot (two slots)
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int RING_BYTES = 192 * 1024;
+constexpr int RING_BYTES = 160 * 1024;     // operand pipeline
+constexpr int STAGING_BYTES = 32 * 1024;   // epilogue transposition buffer, 8 KB per epilogue warp
 constexpr int MAX_STAGES = 6;
+constexpr int META_MAX_BYTES = 24 * 1024;   // shared memory left beside the ring for tile metadata
 constexpr unsigned long long MBAR_WAIT_NS = 2000000000ull;   // 2 s
 
 enum { EPI_HIDDEN = 0, EPI_LOGITS = 1, EPI_BINARY = 2, EPI_CAT = 3 };
@@ -173,6 +175,8 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 struct TcShared {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2];
     uint32_t tmem_base;
+    int off[JS_MAXL + 1];          // start of layer l's tile metadata inside `meta`
+    float bias_s[4][256];          // per epilogue warp: bias of the current tile's columns
 };
 
 // ------------------------------------------------------------------ engine
@@ -183,6 +187,8 @@ struct TcEngine {
     const RunArgs &r;
     TcShared &sh;
     uint8_t *ring;
+    uint8_t *staging;
+    const int *meta;               // tile metadata in shared memory: per layer kb_end[nt], dmin[nt], dmax[nt]
     unsigned epoch = 0;
     unsigned long long issued = 0, skipped = 0;
     int warp, lane;
@@ -194,11 +200,21 @@ struct TcEngine {
     bool dead = false;
     uint32_t tmem_base = 0;
 
-    __device__ TcEngine(const MadeDev &m_, const TcDev &t_, const RunArgs &r_, TcShared &sh_, uint8_t *ring_)
-        : m(m_), t(t_), r(r_), sh(sh_), ring(ring_)
+    __device__ TcEngine(const MadeDev &m_, const TcDev &t_, const RunArgs &r_, TcShared &sh_, uint8_t *ring_,
+                        const int *meta_)
+        : m(m_), t(t_), r(r_), sh(sh_), ring(ring_), staging(ring_ + RING_BYTES), meta(meta_)
     {
         warp = threadIdx.x >> 5;
         lane = threadIdx.x & 31;
+    }
+
+    int phase_no = 0;              // counts gemm phases, for the optional timeline
+    __device__ void trace(int slot) const
+    {
+        if (r.trace == nullptr || phase_no >= JS_TRACE_PHASES) return;
+        if (blockIdx.x != 0 && blockIdx.x != gridDim.x - 1) return;
+        const int who = blockIdx.x == 0 ? 0 : 1;
+        r.trace[((size_t)who * JS_TRACE_PHASES + phase_no) * JS_TRACE_SLOTS + slot] = global_ns();
     }
 
     __device__ bool barrier()
@@ -207,6 +223,7 @@ struct TcEngine {
         fence_proxy_async();
         const bool ok = grid_barrier(r.ctl, epoch, r.spin_limit);
         fence_proxy_async();
+        if (threadIdx.x == 0) trace(5);
         return ok;
     }
 
@@ -231,6 +248,10 @@ struct TcEngine {
         }
     }
 
+    __device__ int kb_end_of(int l, int nt) const { return meta[sh.off[l] + nt]; }
+    __device__ int dmin_of(int l, int nt) const { return meta[sh.off[l] + t.lay[l].nt + nt]; }
+    __device__ int dmax_of(int l, int nt) const { return meta[sh.off[l] + 2 * t.lay[l].nt + nt]; }
+
     __device__ uint8_t *stage_a(int s) const { return ring + (size_t)s * t.stage_bytes; }
     __device__ uint8_t *stage_b(int s) const { return ring + (size_t)s * t.stage_bytes + A_BYTES; }
     __device__ void advance_stage()
@@ -251,10 +272,10 @@ struct TcEngine {
         const int lo_key = is_out ? w.olo + 1 : w.hdeg_lo + 1;   // live iff dmax >= lo_key
         const int hi_key = is_out ? w.ohi : w.hdeg_hi;           // live iff dmin <= hi_key
         int a = 0, b = ly.nt;
-        while (a < b) { const int mid = (a + b) >> 1; if (ly.dmax[mid] >= lo_key) b = mid; else a = mid + 1; }
+        while (a < b) { const int mid = (a + b) >> 1; if (dmax_of(l, mid) >= lo_key) b = mid; else a = mid + 1; }
         nt_lo = a;
         a = nt_lo; b = ly.nt;
-        while (a < b) { const int mid = (a + b) >> 1; if (ly.dmin[mid] > hi_key) b = mid; else a = mid + 1; }
+        while (a < b) { const int mid = (a + b) >> 1; if (dmin_of(l, mid) > hi_key) b = mid; else a = mid + 1; }
         nt_hi = a;
     }
 
@@ -263,9 +284,10 @@ struct TcEngine {
         const TcLayer &ly = t.lay[l];
         const CUtensorMap *ma = t.tmA + l, *mw = t.tmW + l;
         const uint32_t bytes = A_BYTES + ly.bn * BK * 2;
+        trace(0);
         for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
             const int nt = nt_lo + id / MT, mt = id % MT;
-            const int kb_end = ly.kb_end[nt];
+            const int kb_end = kb_end_of(l, nt);
             for (int kb = 0; kb < kb_end; ++kb) {
                 if (!mbar_wait(&sh.empty[stage], sphase ^ 1u, r.ctl)) { dead = true; break; }
                 mbar_expect_tx(&sh.full[stage], bytes);
@@ -282,13 +304,14 @@ struct TcEngine {
         const uint32_t idesc = instr_desc_bf16(ly.bn);
         for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
             const int nt = nt_lo + id / MT;
-            const int kb_end = ly.kb_end[nt];
+            const int kb_end = kb_end_of(l, nt);
             if (!mbar_wait(&sh.tempty[acc], aphase ^ 1u, r.ctl)) { dead = true; break; }
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_COLS);
             for (int kb = 0; kb < kb_end; ++kb) {
                 if (!mbar_wait(&sh.full[stage], sphase, r.ctl)) { dead = true; break; }
                 tc_fence_after();
+                if (kb == 0 && id == (int)blockIdx.x) trace(1);
                 const uint64_t adesc = smem_desc_sw128(smem_u32(stage_a(stage)));
                 const uint64_t bdesc = smem_desc_sw128(smem_u32(stage_b(stage)));
 #pragma unroll
@@ -302,36 +325,10 @@ struct TcEngine {
             umma_commit(&sh.tfull[acc]);                // accumulator complete
             advance_acc();
         }
+        trace(2);
     }
 
-    // ---- epilogues: thread = one sample row of the tile, 32 columns at a time
-    __device__ void epi_hidden(int l, int row, int n0, int c0, const float (&v)[32])
-    {
-        const int N = m.n[l + 1];
-        if (row >= r.batch) return;
-        __nv_bfloat16 *out = (__nv_bfloat16 *)m.a[l + 1] + (size_t)row * N;
-        const float *bias = m.bias[l];
-        const int col = n0 + c0;
-        if (col + 32 <= N) {
-            uint32_t pk[16];
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-                const float4 b4 = __ldg(reinterpret_cast<const float4 *>(bias + col + i));
-                const float f0 = js_act_fn(m.act, v[i] + b4.x), f1 = js_act_fn(m.act, v[i + 1] + b4.y);
-                const float f2 = js_act_fn(m.act, v[i + 2] + b4.z), f3 = js_act_fn(m.act, v[i + 3] + b4.w);
-                pk[i / 2] = pack_bf16x2(f0, f1);
-                pk[i / 2 + 1] = pack_bf16x2(f2, f3);
-            }
-            uint4 *dst = reinterpret_cast<uint4 *>(out + col);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) dst[i] = make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-                if (col + i < N) out[col + i] = __float2bfloat16_rn(js_act_fn(m.act, v[i] + bias[col + i]));
-        }
-    }
-
+    // ---- chunk-wise epilogues: thread = one sample row of the tile, 32 columns at a time
     __device__ void epi_logits(float *zout, int row, int n0, int c0, const float (&v)[32])
     {
         const int N = m.n[m.L + 1];
@@ -341,71 +338,6 @@ struct TcEngine {
 #pragma unroll
         for (int i = 0; i < 32; ++i)
             if (col + i < N) zout[(size_t)row * N + col + i] = v[i] + bias[col + i];
-    }
-
-    // binary positions d = n0 + c0 + i: threshold against the fixed noise, compare, commit
-    __device__ void epi_binary(const Win &w, int row, int n0, int c0, const float (&v)[32], bool &changed,
-                               int &first)
-    {
-        const int T_ = m.T;
-        if (row >= r.batch) return;
-        const int d0 = n0 + c0;
-        if (d0 >= w.phi || d0 + 32 <= w.plo || d0 >= T_) return;
-        const float *bias = m.bias[m.L];
-        const size_t at = (size_t)row * T_ + d0;
-        __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
-        const float lut0 = m.lut[0], lut1 = m.lut[1];
-        if (d0 + 32 <= T_) {
-            uint32_t xo[8], xn[8];
-            const uint2 *xp = reinterpret_cast<const uint2 *>(r.x + at);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { const uint2 u = xp[i]; xo[2 * i] = u.x; xo[2 * i + 1] = u.y; }
-            uint32_t enc[16];
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-                const float4 b4 = __ldg(reinterpret_cast<const float4 *>(bias + d0 + i));
-                const float4 n4 = __ldg(reinterpret_cast<const float4 *>(r.noise + at + i));
-                const float bb[4] = {b4.x, b4.y, b4.z, b4.w}, nn[4] = {n4.x, n4.y, n4.z, n4.w};
-                uint32_t word = 0;
-                float e[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int d = d0 + i + j;
-                    const uint32_t old = (xo[i / 4] >> (8 * j)) & 0xffu;
-                    uint32_t nv = (uint32_t)js_sample_binary(r.nk, v[i + j] + bb[j], nn[j]);
-                    if (d < w.plo || d >= w.phi) nv = old;
-                    if (nv != old) {
-                        if (!changed) first = d;
-                        changed = true;
-                    }
-                    word |= nv << (8 * j);
-                    e[j] = nv ? lut1 : lut0;
-                }
-                xn[i / 4] = word;
-                enc[i / 2] = pack_bf16x2(e[0], e[1]);
-                enc[i / 2 + 1] = pack_bf16x2(e[2], e[3]);
-            }
-            uint2 *xq = reinterpret_cast<uint2 *>(r.x + at);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) xq[i] = make_uint2(xn[2 * i], xn[2 * i + 1]);
-            uint4 *aq = reinterpret_cast<uint4 *>(a0 + at);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) aq[i] = make_uint4(enc[4 * i], enc[4 * i + 1], enc[4 * i + 2], enc[4 * i + 3]);
-        } else {
-#pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const int d = d0 + i;
-                if (d >= T_ || d < w.plo || d >= w.phi) continue;
-                const int old = r.x[at + i];
-                const int nv = js_sample_binary(r.nk, v[i] + bias[d], r.noise[at + i]);
-                if (nv != old) {
-                    if (!changed) first = d;
-                    changed = true;
-                    r.x[at + i] = (uint8_t)nv;
-                    a0[at + i] = __float2bfloat16_rn(nv ? lut1 : lut0);
-                }
-            }
-        }
     }
 
     // one 256-way position per tile: running argmax of logit + Gumbel noise, lowest index wins ties
@@ -427,6 +359,149 @@ struct TcEngine {
         }
     }
 
+
+    // ---- whole-tile epilogues that go through shared memory so that global accesses are
+    // coalesced.  Each epilogue warp owns 32 rows of the tile and an 8 KB staging area holding
+    // 32 rows x 256 bytes; 16-byte chunk c of row r sits at chunk c ^ (r & 15) (conflict-free both
+    // for the row-per-lane writes and for the row-wise reads).
+    __device__ uint8_t *my_staging() const { return staging + (size_t)(warp - 2) * 8192; }
+
+    __device__ void load_bias_tile(int l, int n0, int bn)
+    {
+        float *bs = sh.bias_s[warp - 2];
+        const int N = m.n[l + 1];
+        __syncwarp();
+        for (int i = lane; i < bn; i += 32) bs[i] = (n0 + i < N) ? m.bias[l][n0 + i] : 0.0f;
+        __syncwarp();
+    }
+
+    __device__ void release_acc()
+    {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.tempty[acc]);
+    }
+
+    // hidden layer: act(acc + bias) -> bf16, 128 columns
+    __device__ void epi_hidden_tile(int l, int mt, int n0, uint32_t tbase)
+    {
+        uint8_t *stg = my_staging();
+        const float *bs = sh.bias_s[warp - 2];
+#pragma unroll 1
+        for (int c0 = 0; c0 < 128; c0 += 32) {
+            float v[32];
+            tmem_ld32(tbase + (uint32_t)c0, v);
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 32; i += 2)
+                pk[i / 2] = pack_bf16x2(js_act_fn(m.act, v[i] + bs[c0 + i]), js_act_fn(m.act, v[i + 1] + bs[c0 + i + 1]));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int chunk = c0 / 8 + i;
+                *reinterpret_cast<uint4 *>(stg + lane * 256 + ((chunk ^ (lane & 15)) << 4)) =
+                    make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+            }
+        }
+        release_acc();          // all TMEM reads of this tile are done (and the warp is in step)
+        if (warp == 2 && lane == 0) trace(6);
+        const int N = m.n[l + 1];
+        __nv_bfloat16 *out = (__nv_bfloat16 *)m.a[l + 1];
+        const int q = warp & 3, ch = lane & 15;
+        const int col = n0 + ch * 8;
+#pragma unroll 4
+        for (int it = 0; it < 16; ++it) {
+            const int rl = it * 2 + (lane >> 4);
+            const uint4 val = *reinterpret_cast<const uint4 *>(stg + rl * 256 + ((ch ^ (rl & 15)) << 4));
+            const int row = mt * BM + q * 32 + rl;
+            if (row < r.batch && col < N) *reinterpret_cast<uint4 *>(out + (size_t)row * N + col) = val;
+        }
+        __syncwarp();
+    }
+
+    // binary output layer: 128 positions per tile, handled as two halves of 64
+    __device__ void epi_binary_tile(const Win &w, int mt, int n0, uint32_t tbase, bool flag, int parity,
+                                    bool &wany, int &wfirst)
+    {
+        uint8_t *stg = my_staging();
+        const float *bs = sh.bias_s[warp - 2];
+        const int T_ = m.T, q = warp & 3;
+        __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
+        const float lut0 = m.lut[0], lut1 = m.lut[1];
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+#pragma unroll 1
+            for (int cc = 0; cc < 2; ++cc) {
+                const int c0 = half * 64 + cc * 32;
+                float v[32];
+                tmem_ld32(tbase + (uint32_t)c0, v);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int chunk = cc * 8 + i;
+                    *reinterpret_cast<float4 *>(stg + lane * 256 + ((chunk ^ (lane & 15)) << 4)) =
+                        make_float4(v[4 * i] + bs[c0 + 4 * i], v[4 * i + 1] + bs[c0 + 4 * i + 1],
+                                    v[4 * i + 2] + bs[c0 + 4 * i + 2], v[4 * i + 3] + bs[c0 + 4 * i + 3]);
+                }
+            }
+            if (half == 1) release_acc(); else __syncwarp();
+            const int dbase = n0 + half * 64;
+            const int d = dbase + 2 * lane;                      // this lane's two positions d, d+1
+            const bool half_live = dbase < w.phi && dbase + 64 > w.plo && dbase < T_;
+            if (half_live) {
+                const bool in0 = d >= w.plo && d < w.phi && d < T_;
+                const bool in1 = d + 1 >= w.plo && d + 1 < w.phi && d + 1 < T_;
+#pragma unroll 1
+                for (int g = 0; g < 32; g += 8) {
+                    const int row0 = mt * BM + q * 32 + g;
+                    if (row0 >= r.batch) break;
+                    // issue the loads of eight rows together: the loop is latency-bound otherwise
+                    float2 nz[8];
+                    unsigned short xo[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        nz[j] = make_float2(0.0f, 0.0f);
+                        xo[j] = 0;
+                        if (row0 + j < r.batch && (in0 || in1)) {
+                            const size_t at = (size_t)(row0 + j) * T_ + d;
+                            nz[j] = __ldg(reinterpret_cast<const float2 *>(r.noise + at));
+                            xo[j] = *reinterpret_cast<const unsigned short *>(r.x + at);
+                        }
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        const int rl = g + j, row = row0 + j;
+                        if (row >= r.batch) break;
+                        const float2 z = *reinterpret_cast<const float2 *>(
+                            stg + rl * 256 + ((((lane >> 1) ^ (rl & 15))) << 4) + (lane & 1) * 8);
+                        bool c0 = false, c1 = false;
+                        if (in0 || in1) {
+                            const size_t at = (size_t)row * T_ + d;
+                            const uint32_t o0 = xo[j] & 0xffu, o1 = xo[j] >> 8;
+                            const uint32_t n0v = in0 ? (uint32_t)js_sample_binary(r.nk, z.x, nz[j].x) : o0;
+                            const uint32_t n1v = in1 ? (uint32_t)js_sample_binary(r.nk, z.y, nz[j].y) : o1;
+                            c0 = n0v != o0;
+                            c1 = n1v != o1;
+                            if (c0 || c1) {
+                                *reinterpret_cast<unsigned short *>(r.x + at) = (unsigned short)(n0v | (n1v << 8));
+                                *reinterpret_cast<uint32_t *>(a0 + at) =
+                                    pack_bf16x2(n0v ? lut1 : lut0, n1v ? lut1 : lut0);
+                            }
+                        }
+                        const unsigned bal = __ballot_sync(0xffffffffu, c0 || c1);
+                        if (bal != 0u && flag) {
+                            const int fl = __ffs(bal) - 1;
+                            const int fc0 = __shfl_sync(0xffffffffu, (int)c0, fl);
+                            const int fd = dbase + 2 * fl + (fc0 ? 0 : 1);
+                            if (lane == 0) r.smp_changed[parity * r.batch + row] = 1;
+                            wany = true;
+                            wfirst = min(wfirst, fd);
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+        }
+    }
+
     __device__ void epilogue(int l, int kind, const Win &w, bool flag, int parity, float *zout, int nt_lo,
                              int ntiles, int MT)
     {
@@ -436,43 +511,50 @@ struct TcEngine {
         int first = INT_MAX;
         for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
             const int nt = nt_lo + id / MT, mt = id % MT;
+            if (kind == EPI_HIDDEN || kind == EPI_BINARY) load_bias_tile(l, nt * ly.bn, ly.bn);
             if (!mbar_wait(&sh.tfull[acc], aphase, r.ctl)) { dead = true; break; }
             tc_fence_after();
+            if (warp == 2 && lane == 0) trace(3);
             const int row = mt * BM + q * 32 + lane;
             const int n0 = nt * ly.bn;
             const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS);
-            float best = -INFINITY;
-            int bi = 0;
-            bool ch = false;
-            int fc = INT_MAX;
-            for (int c0 = 0; c0 < ly.bn; c0 += 32) {
-                float v[32];
-                tmem_ld32(tbase + (uint32_t)c0, v);
-                if (kind == EPI_HIDDEN) epi_hidden(l, row, n0, c0, v);
-                else if (kind == EPI_LOGITS) epi_logits(zout, row, n0, c0, v);
-                else if (kind == EPI_BINARY) epi_binary(w, row, n0, c0, v, ch, fc);
-                else epi_cat_chunk(row, nt, c0, v, best, bi);
-            }
-            if (kind == EPI_CAT && row < r.batch && nt >= w.plo && nt < w.phi) {
-                const size_t at = (size_t)row * m.T + nt;
-                if ((int)r.x[at] != bi) {
-                    r.x[at] = (uint8_t)bi;
-                    ((__nv_bfloat16 *)m.a[0])[at] = __float2bfloat16_rn(m.lut[bi]);
-                    ch = true;
-                    fc = nt;
+            if (kind == EPI_HIDDEN) {
+                epi_hidden_tile(l, mt, n0, tbase);
+            } else if (kind == EPI_BINARY) {
+                bool wany = false;
+                int wfirst = INT_MAX;
+                epi_binary_tile(w, mt, n0, tbase, flag, parity, wany, wfirst);
+                if (wany) { any_changed = true; first = min(first, wfirst); }
+            } else {
+                float best = -INFINITY;
+                int bi = 0;
+                bool ch = false;
+                int fc = INT_MAX;
+                for (int c0 = 0; c0 < ly.bn; c0 += 32) {
+                    float v[32];
+                    tmem_ld32(tbase + (uint32_t)c0, v);
+                    if (kind == EPI_LOGITS) epi_logits(zout, row, n0, c0, v);
+                    else epi_cat_chunk(row, nt, c0, v, best, bi);
                 }
+                if (kind == EPI_CAT && row < r.batch && nt >= w.plo && nt < w.phi) {
+                    const size_t at = (size_t)row * m.T + nt;
+                    if ((int)r.x[at] != bi) {
+                        r.x[at] = (uint8_t)bi;
+                        ((__nv_bfloat16 *)m.a[0])[at] = __float2bfloat16_rn(m.lut[bi]);
+                        ch = true;
+                        fc = nt;
+                    }
+                }
+                if (flag && ch) {
+                    r.smp_changed[parity * r.batch + row] = 1;
+                    any_changed = true;
+                    first = min(first, fc);
+                }
+                release_acc();
             }
-            if (flag && ch) {
-                r.smp_changed[parity * r.batch + row] = 1;
-                any_changed = true;
-                first = min(first, fc);
-            }
-            // release the accumulator slot
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh.tempty[acc]);
             advance_acc();
         }
+        if (warp == 2 && lane == 0) trace(4);
         if (flag) {
             const bool wany = __any_sync(0xffffffffu, any_changed);
             if (wany) {
@@ -500,6 +582,7 @@ struct TcEngine {
             if (blockIdx.x == 0) skipped += (unsigned long long)(t.lay[l].nt - nlive) * MT;
         }
         if (ntiles == 0) return false;
+        phase_no++;
         if (warp == 0) {
             if (lane == 0) producer(l, nt_lo, ntiles, MT);
         } else if (warp == 1) {
@@ -546,11 +629,27 @@ made_tc_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ TcDev 
         fence_proxy_async();
     }
     if (warp == 1) tmem_alloc(&sh.tmem_base, 512);
+    // tile metadata of every layer into shared memory (the range searches and the K-loop bounds
+    // would otherwise be chains of dependent global loads in every phase)
+    int *meta = reinterpret_cast<int *>(ring + RING_BYTES + STAGING_BYTES);
+    {
+        int off = 0;
+        for (int l = 0; l <= m.L; ++l) {
+            const int nt = t.lay[l].nt;
+            if (threadIdx.x == 0) sh.off[l] = off;
+            for (int i = threadIdx.x; i < nt; i += blockDim.x) {
+                meta[off + i] = t.lay[l].kb_end[i];
+                meta[off + nt + i] = t.lay[l].dmin[i];
+                meta[off + 2 * nt + i] = t.lay[l].dmax[i];
+            }
+            off += 3 * nt;
+        }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
 
-    TcEngine e(m, t, r, sh, ring);
+    TcEngine e(m, t, r, sh, ring, meta);
     e.tmem_base = sh.tmem_base;
     DriverResult res = made_driver(e, m, r);
     if (e.dead) res.alive = false;
@@ -660,8 +759,16 @@ int js_tc_prepare(js_model *mo)
     t.tmA = (const CUtensorMap *)pa;
     t.tmW = (const CUtensorMap *)pw;
 
-    const int smem = RING_BYTES + 1024;
-    if (cudaFuncSetAttribute(made_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return 0;
+    int meta_ints = 0;
+    for (int l = 0; l <= L; ++l) meta_ints += 3 * t.lay[l].nt;
+    if (meta_ints * 4 > META_MAX_BYTES) return 0;
+    t.smem_bytes = RING_BYTES + STAGING_BYTES + 1024 + ((meta_ints * 4 + 127) & ~127);
+    // the attribute belongs to the function, not to a model: always allow the largest request
+    const int smem = RING_BYTES + STAGING_BYTES + 1024 + META_MAX_BYTES;
+    if (cudaFuncSetAttribute(made_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+        cudaGetLastError();      // not sticky: the CUDA-core kernels will serve this model
+        return 0;
+    }
     int dev = 0, sms = 0, per_sm = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -682,6 +789,6 @@ int js_launch_made_tc(const js_model *mo, const RunArgs &r, cudaStream_t stream)
     const int grid = std::max(1, std::min(mo->tc_max_grid, tiles));
     void *args[3] = {(void *)&v, (void *)&t, (void *)&r};
     cudaError_t e = cudaLaunchCooperativeKernel((const void *)made_tc_kernel, dim3(grid), dim3(NTH), args,
-                                                RING_BYTES + 1024, stream);
+                                                t.smem_bytes, stream);
     return e == cudaSuccess ? 0 : (int)e;
 }
