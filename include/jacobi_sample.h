@@ -148,6 +148,7 @@ typedef struct {
     long long tiles_skipped;   /* output tiles skipped as final, finished or masked */
     int path;                  /* 0 tensor-core kernels, 1 CUDA-core kernels */
     int status;                /* the call's return value */
+    int compactions;           /* times finished samples were moved out of the working batch */
 } js_stats;
 int js_get_stats(const js_model *m, js_stats *out);
 

@@ -162,6 +162,7 @@ int common_scratch(js_model *m, int T)
     if ((rc = dev_alloc<JsCtl>(m, &m->ctl, 1, true)) != JS_OK) return rc;
     if ((rc = dev_alloc<int>(m, &m->smp_changed, 2 * (size_t)m->rows, true)) != JS_OK) return rc;
     if ((rc = dev_alloc<int>(m, &m->smp_state, 2 * (size_t)m->rows, true)) != JS_OK) return rc;
+    if ((rc = dev_alloc<int>(m, &m->perm, 2 * (size_t)m->rows, true)) != JS_OK) return rc;
     if ((rc = dev_alloc<uint8_t>(m, &m->x_old, (size_t)m->rows * T, true)) != JS_OK) return rc;
     if ((rc = dev_alloc<uint8_t>(m, &m->x_tmp, (size_t)m->rows * T, true)) != JS_OK) return rc;
     if ((rc = dev_alloc<unsigned long long>(m, &m->trace, 2 * JS_TRACE_PHASES * JS_TRACE_SLOTS, true)) != JS_OK) return rc;
@@ -185,6 +186,9 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
     r.x_old = m->x_old;
     r.frontier_skip = m->opt_frontier_skip;
     r.seq_skip = m->opt_seq_skip;
+    r.compact = m->opt_compact;
+    r.perm = m->perm;
+    r.perm_stride = m->rows;
     r.spin_limit = (unsigned)m->opt_spin_limit;
     r.trace = m->opt_trace ? m->trace : nullptr;
     if (r.trace) CU_TRY(cudaMemsetAsync(m->trace, 0, sizeof(unsigned long long) * 2 * JS_TRACE_PHASES * JS_TRACE_SLOTS, st));
@@ -225,6 +229,7 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
     m->stats.tiles_skipped = (long long)h.tiles_skipped;
     m->stats.batch_iters_max = h.iters_max;
     m->stats.path = used_path;
+    m->stats.compactions = h.compactions;
     m->stats.status = h.status;
     return h.status;
 }

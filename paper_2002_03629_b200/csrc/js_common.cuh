@@ -26,6 +26,7 @@ struct JsCtl {
     int frontier;           // leading positions known final at exit
     int iters_max;
     int live;               // samples still iterating (tensor-core path)
+    int compactions;        // times the working batch was compacted
     unsigned long long tiles_issued, tiles_skipped;
 };
 
@@ -60,7 +61,9 @@ struct RunArgs {
     int *smp_state;           // [2][batch] per-sample bookkeeping (done flag, running count)
     const uint8_t *x_in;      // KM_FORWARD: symbols
     float *logits_out;        // KM_FORWARD: destination
-    int frontier_skip, seq_skip;
+    int *perm;                // [2][perm_stride]: working row -> sample index, by compaction parity
+    int perm_stride;
+    int frontier_skip, seq_skip, compact;
     unsigned spin_limit;
     JsCtl *ctl;
     unsigned long long *trace;   // [2 CTAs][JS_TRACE_PHASES][JS_TRACE_SLOTS] globaltimer stamps, or NULL

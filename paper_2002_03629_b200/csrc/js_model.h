@@ -31,7 +31,7 @@ struct js_model {
     std::vector<void *> allocs;   // every device allocation, freed by js_model_destroy
     std::vector<std::vector<int>> host_deg;
     JsCtl *ctl = nullptr;
-    int *smp_changed = nullptr, *smp_state = nullptr;
+    int *smp_changed = nullptr, *smp_state = nullptr, *perm = nullptr;
     uint8_t *x_old = nullptr, *x_tmp = nullptr;
     unsigned long long *trace = nullptr;
     int opt_frontier_skip = 1, opt_seq_skip = 0, opt_spin_limit = 1 << 22, opt_path = 0, opt_compact = 1, opt_trace = 0;

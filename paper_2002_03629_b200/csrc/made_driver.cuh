@@ -120,6 +120,13 @@ __device__ DriverResult made_driver(E &e, const MadeDev &m, const RunArgs &r)
                 if (any && cap < T_) res.status = JS_NOT_CONVERGED;
                 break;
             }
+            // samples that stopped changing are at their fixed point: drop them from the working
+            // batch when that frees a whole tile of rows (hidden rows are then recomputed)
+            if (r.compact) {
+                const int c = e.compact(p);
+                if (c < 0) { res.alive = false; return res; }
+                if (c > 0) fin_h = 0;
+            }
         }
         res.frontier = fin_x;
         return res;

@@ -357,6 +357,7 @@ struct GenericEngine {
     }
     __device__ bool barrier() { return grid_barrier(r.ctl, epoch, r.spin_limit); }
     __device__ void init(const uint8_t *src) { init_phase<T>(m, r, src); }
+    __device__ int compact(int) { return 0; }      // the CUDA-core path keeps the batch as it is
     __device__ bool forward_logits(float *zout)
     {
         const Win w = make_win(0, m.T, 0, m.T);

@@ -177,6 +177,8 @@ struct TcShared {
     uint32_t tmem_base;
     int off[JS_MAXL + 1];          // start of layer l's tile metadata inside `meta`
     float bias_s[4][256];          // per epilogue warp: bias of the current tile's columns
+    int wcnt[NTH / 32];            // compaction: per-warp counts
+    int cbase;                     // compaction: rows kept so far
 };
 
 // ------------------------------------------------------------------ engine
@@ -199,6 +201,9 @@ struct TcEngine {
     uint32_t aphase = 0;
     bool dead = false;
     uint32_t tmem_base = 0;
+    // working batch: rows [0, live) of the activation buffers hold samples perm[pcur][row]
+    int live = 0;
+    int pcur = 0;
 
     __device__ TcEngine(const MadeDev &m_, const TcDev &t_, const RunArgs &r_, TcShared &sh_, uint8_t *ring_,
                         const int *meta_)
@@ -206,7 +211,9 @@ struct TcEngine {
     {
         warp = threadIdx.x >> 5;
         lane = threadIdx.x & 31;
+        live = r.batch;
     }
+    __device__ const int *perm_cur() const { return r.perm + (size_t)pcur * r.perm_stride; }
 
     int phase_no = 0;              // counts gemm phases, for the optional timeline
     __device__ void trace(int slot) const
@@ -241,11 +248,62 @@ struct TcEngine {
                 r.smp_changed[i] = 0;
                 r.smp_state[i] = 0;
             }
+            for (int i = threadIdx.x; i < r.batch; i += blockDim.x) r.perm[i] = i;
             if (threadIdx.x == 0) {
                 r.ctl->agg_any[0] = r.ctl->agg_any[1] = 0;
                 r.ctl->agg_minfirst[0] = r.ctl->agg_minfirst[1] = INT_MAX;
             }
         }
+    }
+
+    // Compaction of the working batch after an iteration of parity `parity`.  Every CTA computes
+    // the same list (rows whose sample changed, in order) from the per-sample flags, so no exchange
+    // is needed to agree on it.  It is adopted only when it frees at least one 128-row tile; then
+    // the encoded iterate is rebuilt for the new rows and a grid barrier makes it visible.
+    // Returns 1 if rows were remapped, 0 if not, -1 if the barrier gave up.
+    __device__ int compact(int parity)
+    {
+        const int *pc = perm_cur();
+        int *pn = r.perm + (size_t)(pcur ^ 1) * r.perm_stride;
+        const int *chg = r.smp_changed + (size_t)parity * r.batch;
+        if (threadIdx.x == 0) sh.cbase = 0;
+        __syncthreads();
+        for (int base = 0; base < live; base += NTH) {
+            const int row = base + threadIdx.x;
+            int b = -1;
+            bool keep = false;
+            if (row < live) {
+                b = pc[row];
+                keep = ld_volatile_i32(&chg[b]) != 0;
+            }
+            const unsigned bal = __ballot_sync(0xffffffffu, keep);
+            if (lane == 0) sh.wcnt[warp] = __popc(bal);
+            __syncthreads();
+            int off = sh.cbase;
+            for (int w2 = 0; w2 < warp; ++w2) off += sh.wcnt[w2];
+            if (keep) pn[off + __popc(bal & ((1u << lane) - 1u))] = b;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                int tot = 0;
+                for (int w2 = 0; w2 < NTH / 32; ++w2) tot += sh.wcnt[w2];
+                sh.cbase += tot;
+            }
+            __syncthreads();
+        }
+        const int nlive = sh.cbase;
+        __syncthreads();
+        if ((nlive + BM - 1) / BM >= (live + BM - 1) / BM) return 0;
+        live = nlive;
+        pcur ^= 1;
+        if (blockIdx.x == 0 && threadIdx.x == 0) { r.ctl->compactions += 1; r.ctl->live = nlive; }
+        __threadfence_block();
+        __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
+        const size_t n = (size_t)live * m.T;
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+            const int row = (int)(i / m.T), d = (int)(i % m.T);
+            a0[i] = __float2bfloat16_rn(m.lut[r.x[(size_t)pn[row] * m.T + d]]);
+        }
+        return barrier() ? 1 : -1;
     }
 
     __device__ int kb_end_of(int l, int nt) const { return meta[sh.off[l] + nt]; }
@@ -341,11 +399,11 @@ struct TcEngine {
     }
 
     // one 256-way position per tile: running argmax of logit + Gumbel noise, lowest index wins ties
-    __device__ void epi_cat_chunk(int row, int d, int c0, const float (&v)[32], float &best, int &bi)
+    __device__ void epi_cat_chunk(int sample, int d, int c0, const float (&v)[32], float &best, int &bi)
     {
-        if (row >= r.batch) return;
+        if (sample < 0) return;
         const float *bias = m.bias[m.L] + (size_t)d * 256 + c0;
-        const float *gg = r.noise + ((size_t)row * m.T + d) * 256 + c0;
+        const float *gg = r.noise + ((size_t)sample * m.T + d) * 256 + c0;
 #pragma unroll
         for (int i = 0; i < 32; i += 4) {
             const float4 b4 = __ldg(reinterpret_cast<const float4 *>(bias + i));
@@ -413,7 +471,7 @@ struct TcEngine {
             const int rl = it * 2 + (lane >> 4);
             const uint4 val = *reinterpret_cast<const uint4 *>(stg + rl * 256 + ((ch ^ (rl & 15)) << 4));
             const int row = mt * BM + q * 32 + rl;
-            if (row < r.batch && col < N) *reinterpret_cast<uint4 *>(out + (size_t)row * N + col) = val;
+            if (row < live && col < N) *reinterpret_cast<uint4 *>(out + (size_t)row * N + col) = val;
         }
         __syncwarp();
     }
@@ -427,6 +485,7 @@ struct TcEngine {
         const int T_ = m.T, q = warp & 3;
         __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
         const float lut0 = m.lut[0], lut1 = m.lut[1];
+        const int *pm = perm_cur();
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
 #pragma unroll 1
@@ -452,16 +511,19 @@ struct TcEngine {
 #pragma unroll 1
                 for (int g = 0; g < 32; g += 8) {
                     const int row0 = mt * BM + q * 32 + g;
-                    if (row0 >= r.batch) break;
+                    if (row0 >= live) break;
                     // issue the loads of eight rows together: the loop is latency-bound otherwise
+                    int sb[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) sb[j] = row0 + j < live ? pm[row0 + j] : 0;
                     float2 nz[8];
                     unsigned short xo[8];
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         nz[j] = make_float2(0.0f, 0.0f);
                         xo[j] = 0;
-                        if (row0 + j < r.batch && (in0 || in1)) {
-                            const size_t at = (size_t)(row0 + j) * T_ + d;
+                        if (row0 + j < live && (in0 || in1)) {
+                            const size_t at = (size_t)sb[j] * T_ + d;
                             nz[j] = __ldg(reinterpret_cast<const float2 *>(r.noise + at));
                             xo[j] = *reinterpret_cast<const unsigned short *>(r.x + at);
                         }
@@ -469,12 +531,12 @@ struct TcEngine {
 #pragma unroll
                     for (int j = 0; j < 8; ++j) {
                         const int rl = g + j, row = row0 + j;
-                        if (row >= r.batch) break;
+                        if (row >= live) break;
                         const float2 z = *reinterpret_cast<const float2 *>(
                             stg + rl * 256 + ((((lane >> 1) ^ (rl & 15))) << 4) + (lane & 1) * 8);
                         bool c0 = false, c1 = false;
                         if (in0 || in1) {
-                            const size_t at = (size_t)row * T_ + d;
+                            const size_t at = (size_t)sb[j] * T_ + d;
                             const uint32_t o0 = xo[j] & 0xffu, o1 = xo[j] >> 8;
                             const uint32_t n0v = in0 ? (uint32_t)js_sample_binary(r.nk, z.x, nz[j].x) : o0;
                             const uint32_t n1v = in1 ? (uint32_t)js_sample_binary(r.nk, z.y, nz[j].y) : o1;
@@ -482,7 +544,7 @@ struct TcEngine {
                             c1 = n1v != o1;
                             if (c0 || c1) {
                                 *reinterpret_cast<unsigned short *>(r.x + at) = (unsigned short)(n0v | (n1v << 8));
-                                *reinterpret_cast<uint32_t *>(a0 + at) =
+                                *reinterpret_cast<uint32_t *>(a0 + (size_t)row * T_ + d) =
                                     pack_bf16x2(n0v ? lut1 : lut0, n1v ? lut1 : lut0);
                             }
                         }
@@ -491,7 +553,7 @@ struct TcEngine {
                             const int fl = __ffs(bal) - 1;
                             const int fc0 = __shfl_sync(0xffffffffu, (int)c0, fl);
                             const int fd = dbase + 2 * fl + (fc0 ? 0 : 1);
-                            if (lane == 0) r.smp_changed[parity * r.batch + row] = 1;
+                            if (lane == 0) r.smp_changed[parity * r.batch + sb[j]] = 1;
                             wany = true;
                             wfirst = min(wfirst, fd);
                         }
@@ -530,23 +592,24 @@ struct TcEngine {
                 int bi = 0;
                 bool ch = false;
                 int fc = INT_MAX;
+                const int sample = (kind == EPI_CAT && row < live) ? perm_cur()[row] : -1;
                 for (int c0 = 0; c0 < ly.bn; c0 += 32) {
                     float v[32];
                     tmem_ld32(tbase + (uint32_t)c0, v);
                     if (kind == EPI_LOGITS) epi_logits(zout, row, n0, c0, v);
-                    else epi_cat_chunk(row, nt, c0, v, best, bi);
+                    else epi_cat_chunk(sample, nt, c0, v, best, bi);
                 }
-                if (kind == EPI_CAT && row < r.batch && nt >= w.plo && nt < w.phi) {
-                    const size_t at = (size_t)row * m.T + nt;
+                if (sample >= 0 && nt >= w.plo && nt < w.phi) {
+                    const size_t at = (size_t)sample * m.T + nt;
                     if ((int)r.x[at] != bi) {
                         r.x[at] = (uint8_t)bi;
-                        ((__nv_bfloat16 *)m.a[0])[at] = __float2bfloat16_rn(m.lut[bi]);
+                        ((__nv_bfloat16 *)m.a[0])[(size_t)row * m.T + nt] = __float2bfloat16_rn(m.lut[bi]);
                         ch = true;
                         fc = nt;
                     }
                 }
                 if (flag && ch) {
-                    r.smp_changed[parity * r.batch + row] = 1;
+                    r.smp_changed[parity * r.batch + sample] = 1;
                     any_changed = true;
                     first = min(first, fc);
                 }
@@ -572,7 +635,7 @@ struct TcEngine {
     {
         int nt_lo, nt_hi;
         live_range(l, w, nt_lo, nt_hi);
-        const int MT = (r.batch + BM - 1) / BM;
+        const int MT = (live + BM - 1) / BM;
         const int nlive = max(0, nt_hi - nt_lo);
         const int ntiles = nlive * MT;
         if (threadIdx.x == 0) {

@@ -190,6 +190,28 @@ def test_max_iters_returns_last_iterate(name):
     np.testing.assert_array_equal(it[exact], it_ref[exact])
 
 
+def test_compaction_changes_nothing_but_the_work():
+    """Finished samples leave the working batch (tensor-core kernels): same samples, same
+    per-sample counts, fewer tiles."""
+    if _path["v"] != 0:
+        pytest.skip("compaction lives in the tensor-core kernels")
+    c = case("chain")
+    p = c.p
+    res = {}
+    for on in (1, 0):
+        c.model.set_option(p.JS_OPT_COMPACT, on)
+        rc, x, it = c.run(p.JS_JACOBI)
+        st = c.model.stats()
+        res[on] = (x, it, st.compactions, st.tiles_issued)
+        assert rc == 0
+    c.model.set_option(p.JS_OPT_COMPACT, 1)
+    np.testing.assert_array_equal(res[1][0], res[0][0])
+    np.testing.assert_array_equal(res[1][1], res[0][1])
+    assert res[0][2] == 0 and res[1][2] >= 1, "the 130-sample case must drop to one row tile at some point"
+    assert res[1][3] < res[0][3]
+    check_samples(c.orc, res[1][0], c.xstar, c.noise, c.nk)
+
+
 def test_examples_of_section_4_on_device():
     """Markov chain (Example 3): T iterations; independent chain (Example 1): one plus the confirmation."""
     p = pkg()
