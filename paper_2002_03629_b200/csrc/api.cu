@@ -180,6 +180,7 @@ bool noise_kind_ok(const js_model *m, int nk)
 int run_made(js_model *m, RunArgs &r, cudaStream_t st)
 {
     const MadeDev &v = m->made;
+    if (m->kind == 1 && r.kmode == KM_JACOBI_GS) return JS_ERR_UNSUPPORTED;
     r.ctl = m->ctl;
     r.smp_changed = m->smp_changed;
     r.smp_state = m->smp_state;
@@ -198,7 +199,11 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
     int rc_launch;
     // the tensor-core epilogues use 16-byte vector accesses on the caller's buffers
     const bool aligned = (((uintptr_t)r.noise | (uintptr_t)r.x | (uintptr_t)r.logits_out) & 15u) == 0;
-    if (m->tc_ok && m->opt_path == 0 && r.kmode != KM_JACOBI_GS && aligned) {
+    if (m->kind == 1) {
+        if (!aligned) return JS_ERR_ARG;
+        used_path = 0;
+        rc_launch = js_launch_conv_tc(m, r, st);
+    } else if (m->tc_ok && m->opt_path == 0 && r.kmode != KM_JACOBI_GS && aligned) {
         used_path = 0;
         rc_launch = js_launch_made_tc(m, r, st);
     } else {
@@ -271,9 +276,27 @@ int js_made_create(const js_made_desc *d, js_model **out)
 
 int js_conv_create(const js_conv_desc *d, js_model **out)
 {
-    (void)d;
-    if (out) *out = nullptr;
-    return JS_ERR_UNSUPPORTED;
+    if (!d || !out) return JS_ERR_ARG;
+    *out = nullptr;
+    if (!d->W || !d->b || !d->lut || d->max_batch < 1 || d->n_conv < 1 || d->n_conv > JS_MAXL) return JS_ERR_ARG;
+    for (int l = 0; l <= d->n_conv; ++l)
+        if (!d->W[l] || !d->b[l]) return JS_ERR_ARG;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "no CUDA device");
+        return JS_ERR_CUDA;
+    }
+    js_model *m = new (std::nothrow) js_model();
+    if (!m) return JS_ERR_ARG;
+    m->kind = 1;
+    m->max_batch = d->max_batch;
+    m->rows = d->max_batch;
+    int rc = js_conv_build(m, d);
+    if (rc == JS_ERR_CUDA) snprintf(g_cuda_err, sizeof g_cuda_err, "conv model: %s", cudaGetErrorString(cudaGetLastError()));
+    if (rc == JS_OK) rc = common_scratch(m, m->conv.T);
+    if (rc != JS_OK) { js_model_destroy(m); return rc; }
+    *out = m;
+    return JS_OK;
 }
 
 void js_model_destroy(js_model *m)
@@ -293,7 +316,6 @@ int jacobi_sample(const js_model *cm, int batch, const float *noise_dev, int nk,
     if (!noise_kind_ok(m, nk)) return JS_ERR_ARG;
     const int T = m->kind == 0 ? m->made.T : m->conv_T;
     if ((mode == JS_GS_JACOBI || mode == JS_JACOBI_GS) && (block < 1 || block > T)) return JS_ERR_ARG;
-    if (m->kind != 0) return JS_ERR_UNSUPPORTED;
     RunArgs r;
     memset(&r, 0, sizeof r);
     r.batch = batch; r.noise = noise_dev; r.nk = nk; r.init = init_dev;
@@ -312,7 +334,6 @@ int sequential_sample(const js_model *cm, int batch, const float *noise_dev, int
     if (!m || !noise_dev || !out_samples_dev) return JS_ERR_ARG;
     if (batch < 1 || batch > m->max_batch) return JS_ERR_ARG;
     if (!noise_kind_ok(m, nk)) return JS_ERR_ARG;
-    if (m->kind != 0) return JS_ERR_UNSUPPORTED;
     RunArgs r;
     memset(&r, 0, sizeof r);
     r.batch = batch; r.noise = noise_dev; r.nk = nk; r.kmode = KM_SEQ;
@@ -325,7 +346,6 @@ int js_forward_logits(const js_model *cm, int batch, const uint8_t *x_dev, float
     js_model *m = const_cast<js_model *>(cm);
     if (!m || !x_dev || !logits_dev) return JS_ERR_ARG;
     if (batch < 1 || batch > m->max_batch) return JS_ERR_ARG;
-    if (m->kind != 0) return JS_ERR_UNSUPPORTED;
     RunArgs r;
     memset(&r, 0, sizeof r);
     r.batch = batch; r.kmode = KM_FORWARD; r.x_in = x_dev; r.logits_out = logits_dev;

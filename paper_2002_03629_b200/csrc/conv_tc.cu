@@ -1,0 +1,583 @@
+// Masked-convolution sampler (PixelCNN-style stack) on the sm_100a tensor cores.
+//
+// Every masked 3x3 convolution is an implicit GEMM: M = 128 consecutive pixels of one
+// image (whole rows), N = output channels, K = live taps x input channels.  Only the
+// five taps the causal mask keeps are visited (row above: left, centre, right; same
+// row: left, centre); the centre tap's colour-group mask is already folded into the
+// packed weights.  The A operand of tap (ky, kx) is the activation tensor shifted by
+// (ky-1, kx-1): one 4-D TMA box {64 channels, width, rows, 1 image} whose start
+// coordinate may lie outside the image, where TMA fills zeros - that is the zero
+// padding.  The 1x1 head is a plain GEMM with one 256-class sub-pixel per N tile, and
+// its epilogue is the sampling step (Gumbel-max against the fixed noise, compare,
+// re-encode), as in the masked-MLP kernel.  Solver loops: made_driver.cuh.
+#include <cuda.h>
+
+#include <vector>
+
+#include "js_common.cuh"
+#include "js_model.h"
+#include "made_driver.cuh"
+#include "tc_common.cuh"
+
+namespace {
+
+constexpr int BM = TC_BM, BK = TC_BK;
+constexpr int NTH = 192;
+constexpr int ACC_COLS = 256;
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + 256 * BK * 2;   // A tile + up to 256 weight rows
+constexpr int N_STAGES = 3;
+constexpr int RING_BYTES = N_STAGES * STAGE_BYTES;    // 144 KB
+constexpr int STAGING_BYTES = 32 * 1024;
+constexpr int SMEM_BYTES = RING_BYTES + STAGING_BYTES + 1024;
+constexpr int MAX_IMAGES = 256;
+
+enum { EPI_HIDDEN = 0, EPI_LOGITS = 1, EPI_CAT = 3 };
+
+// the five taps a causal 3x3 kernel keeps, in the order the packed weights use
+__device__ __constant__ int c_tap_ky[5] = {0, 0, 0, 1, 1};
+__device__ __constant__ int c_tap_kx[5] = {0, 1, 2, 0, 1};
+
+struct ConvShared {
+    uint64_t full[N_STAGES], empty[N_STAGES], tfull[2], tempty[2];
+    uint32_t tmem_base;
+    float bias_s[4][256];
+    int img[MAX_IMAGES];      // images still iterating
+    int n_img;
+};
+
+struct ConvEngine {
+    static constexpr bool has_jgs = false;
+    const ConvDev &m;
+    const RunArgs &r;
+    ConvShared &sh;
+    uint8_t *ring, *staging;
+    unsigned epoch = 0;
+    unsigned long long issued = 0, skipped = 0;
+    int warp, lane;
+    int stage = 0;
+    uint32_t sphase = 0;
+    int acc = 0;
+    uint32_t aphase = 0;
+    bool dead = false;
+    uint32_t tmem_base = 0;
+
+    __device__ ConvEngine(const ConvDev &m_, const RunArgs &r_, ConvShared &sh_, uint8_t *ring_)
+        : m(m_), r(r_), sh(sh_), ring(ring_), staging(ring_ + RING_BYTES)
+    {
+        warp = threadIdx.x >> 5;
+        lane = threadIdx.x & 31;
+    }
+
+    __device__ bool barrier()
+    {
+        fence_proxy_async();      // epilogue stores are read by the next layer's TMA loads
+        const bool ok = grid_barrier(r.ctl, epoch, r.spin_limit);
+        fence_proxy_async();
+        return ok;
+    }
+
+    __device__ void init(const uint8_t *src)
+    {
+        const size_t n = (size_t)r.batch * m.T;
+        __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.act[0];
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+            const uint8_t v = src ? src[i] : (uint8_t)0;
+            if (r.x) r.x[i] = v;
+            const size_t pix = i / m.in_ch;                 // global pixel index (image-major)
+            a0[pix * 64 + (i % m.in_ch)] = __float2bfloat16_rn(m.lut[v]);
+        }
+        if (blockIdx.x == 0) {
+            for (int i = threadIdx.x; i < 2 * r.batch; i += blockDim.x) {
+                r.smp_changed[i] = 0;
+                r.smp_state[i] = 0;
+            }
+            if (threadIdx.x == 0) {
+                r.ctl->agg_any[0] = r.ctl->agg_any[1] = 0;
+                r.ctl->agg_minfirst[0] = r.ctl->agg_minfirst[1] = INT_MAX;
+            }
+        }
+        for (int i = threadIdx.x; i < r.batch; i += blockDim.x) sh.img[i] = i;
+        if (threadIdx.x == 0) sh.n_img = r.batch;
+        __syncthreads();
+    }
+
+    // Images whose iterate did not change are at their fixed point: they drop out of the
+    // tile lists.  Every CTA derives the same list from the per-sample flags; rows do not
+    // move, so nothing has to be rebuilt.  Always returns 0 (no remapping).
+    __device__ int compact(int parity)
+    {
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int k = 0;
+            for (int i = 0; i < sh.n_img; ++i) {
+                const int b = sh.img[i];
+                if (ld_volatile_i32(&r.smp_changed[parity * r.batch + b]) != 0) sh.img[k++] = b;
+            }
+            sh.n_img = k;
+            if (blockIdx.x == 0) { r.ctl->compactions += 1; r.ctl->live = k; }
+        }
+        __syncthreads();
+        return 0;
+    }
+
+    __device__ uint8_t *stage_a(int s) const { return ring + (size_t)s * STAGE_BYTES; }
+    __device__ uint8_t *stage_b(int s) const { return ring + (size_t)s * STAGE_BYTES + A_BYTES; }
+    __device__ void advance_stage()
+    {
+        if (++stage == N_STAGES) { stage = 0; sphase ^= 1u; }
+    }
+    __device__ void advance_acc()
+    {
+        acc ^= 1;
+        if (acc == 0) aphase ^= 1u;
+    }
+
+    // row tiles (of every image) that the window touches.  A hidden unit of colour group g at
+    // pixel p reads positions < 3p + g ("degree"); position t = 3p + c.
+    __device__ void live_rows(bool head, const Win &w, int &yt_lo, int &yt_hi) const
+    {
+        const int lo_key = head ? w.olo : w.hdeg_lo + 1;      // live iff largest degree/position >= lo_key
+        const int hi_key = head ? w.ohi - 1 : w.hdeg_hi;      // live iff smallest degree/position <= hi_key
+        yt_lo = m.nyt;
+        yt_hi = 0;
+        for (int yt = 0; yt < m.nyt; ++yt) {
+            const int p0 = yt * m.R * m.width;
+            const int p1 = min(m.height, (yt + 1) * m.R) * m.width - 1;
+            const int dmin = p0 * m.in_ch, dmax = p1 * m.in_ch + m.in_ch - 1;
+            if (dmax >= lo_key && dmin <= hi_key) { yt_lo = min(yt_lo, yt); yt_hi = max(yt_hi, yt + 1); }
+        }
+        if (yt_hi < yt_lo) yt_lo = yt_hi = 0;
+    }
+
+    // tile id -> (image, row tile, sub-pixel); `per` = 1 for conv layers, in_ch for the head
+    __device__ void locate(int id, int nyl, int yt_lo, int per, int &n, int &yt, int &c) const
+    {
+        c = id % per;
+        const int t2 = id / per;
+        yt = yt_lo + t2 % nyl;
+        n = sh.img[t2 / nyl];
+    }
+
+    __device__ int kblocks(int l) const
+    {
+        return l < m.n_conv ? 5 * (m.cin_pad[l] / BK) : m.ch / BK;
+    }
+
+    __device__ void producer(int l, int yt_lo, int nyl, int ntiles)
+    {
+        const bool head = (l == m.n_conv);
+        const int per = head ? m.in_ch : 1;
+        const int bn = head ? 256 : m.ch;
+        const CUtensorMap *ma = m.tmAct + l, *mw = m.tmW + l;
+        const uint32_t bytes = A_BYTES + bn * BK * 2;
+        const int kcs = head ? m.ch / BK : m.cin_pad[l] / BK;
+        for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
+            int n, yt, c;
+            locate(id, nyl, yt_lo, per, n, yt, c);
+            const int y0 = yt * m.R;
+            const int ntaps = head ? 1 : 5;
+            for (int tap = 0; tap < ntaps && !dead; ++tap) {
+                const int dy = head ? 0 : c_tap_ky[tap] - 1, dx = head ? 0 : c_tap_kx[tap] - 1;
+                for (int kc = 0; kc < kcs; ++kc) {
+                    if (!mbar_wait(&sh.empty[stage], sphase ^ 1u, r.ctl)) { dead = true; break; }
+                    mbar_expect_tx(&sh.full[stage], bytes);
+                    tma_load_4d(smem_u32(stage_a(stage)), ma, &sh.full[stage], kc * BK, dx, y0 + dy, n);
+                    tma_load_2d(smem_u32(stage_b(stage)), mw, &sh.full[stage], kc * BK,
+                                head ? c * 256 : tap * m.ch);
+                    advance_stage();
+                }
+            }
+        }
+    }
+
+    __device__ void mma_issuer(int l, int ntiles)
+    {
+        const bool head = (l == m.n_conv);
+        const uint32_t idesc = instr_desc_bf16(head ? 256 : m.ch);
+        const int nkb = kblocks(l);
+        for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
+            if (!mbar_wait(&sh.tempty[acc], aphase ^ 1u, r.ctl)) { dead = true; break; }
+            tc_fence_after();
+            const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_COLS);
+            for (int kb = 0; kb < nkb; ++kb) {
+                if (!mbar_wait(&sh.full[stage], sphase, r.ctl)) { dead = true; break; }
+                tc_fence_after();
+                const uint64_t adesc = smem_desc_sw128(smem_u32(stage_a(stage)));
+                const uint64_t bdesc = smem_desc_sw128(smem_u32(stage_b(stage)));
+#pragma unroll
+                for (int k = 0; k < BK / 16; ++k)
+                    umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                              (kb > 0 || k > 0) ? 1u : 0u);
+                umma_commit(&sh.empty[stage]);
+                advance_stage();
+            }
+            if (dead) break;
+            umma_commit(&sh.tfull[acc]);
+            advance_acc();
+        }
+    }
+
+    __device__ void release_acc()
+    {
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.tempty[acc]);
+    }
+
+    // conv layer: ReLU(acc + bias) -> bf16, through the staging buffer so that the NHWC stores
+    // are coalesced (see the masked-MLP kernel for the layout of the staging rows)
+    __device__ void epi_hidden_tile(int l, int n, int y0, uint32_t tbase)
+    {
+        uint8_t *stg = staging + (size_t)(warp - 2) * 8192;
+        const float *bs = sh.bias_s[warp - 2];
+        const int bn = m.ch;
+#pragma unroll 1
+        for (int c0 = 0; c0 < bn; c0 += 32) {
+            float v[32];
+            tmem_ld32(tbase + (uint32_t)c0, v);
+            uint32_t pk[16];
+#pragma unroll
+            for (int i = 0; i < 32; i += 2)
+                pk[i / 2] = pack_bf16x2(fmaxf(v[i] + bs[c0 + i], 0.0f), fmaxf(v[i + 1] + bs[c0 + i + 1], 0.0f));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int chunk = c0 / 8 + i;
+                *reinterpret_cast<uint4 *>(stg + lane * 256 + ((chunk ^ (lane & 15)) << 4)) =
+                    make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
+            }
+        }
+        release_acc();
+        __nv_bfloat16 *out = (__nv_bfloat16 *)m.act[l + 1];
+        const int q = warp & 3, ch = lane & 15;
+        const int col = ch * 8;
+        const int rows_valid = (min(m.height, y0 + m.R) - y0) * m.width;     // pixels of the tile inside the image
+        const size_t pix0 = (size_t)n * m.height * m.width + (size_t)y0 * m.width;
+#pragma unroll 4
+        for (int it = 0; it < 16; ++it) {
+            const int rl = it * 2 + (lane >> 4);
+            const uint4 val = *reinterpret_cast<const uint4 *>(stg + rl * 256 + ((ch ^ (rl & 15)) << 4));
+            const int prow = q * 32 + rl;
+            if (prow < rows_valid && col < bn) *reinterpret_cast<uint4 *>(out + (pix0 + prow) * bn + col) = val;
+        }
+        __syncwarp();
+    }
+
+    __device__ void epilogue(int l, int kind, const Win &w, bool flag, int parity, float *zout, int yt_lo, int nyl,
+                             int ntiles)
+    {
+        const bool head = (l == m.n_conv);
+        const int per = head ? m.in_ch : 1;
+        const int q = warp & 3;
+        bool any_changed = false;
+        int first = INT_MAX;
+        for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
+            int n, yt, c;
+            locate(id, nyl, yt_lo, per, n, yt, c);
+            const int y0 = yt * m.R;
+            if (!head) {
+                float *bs = sh.bias_s[warp - 2];
+                __syncwarp();
+                for (int i = lane; i < m.ch; i += 32) bs[i] = m.bias[l][i];
+                __syncwarp();
+            }
+            if (!mbar_wait(&sh.tfull[acc], aphase, r.ctl)) { dead = true; break; }
+            tc_fence_after();
+            const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS);
+            if (!head) {
+                epi_hidden_tile(l, n, y0, tbase);
+            } else {
+                // thread = one pixel of the tile; 256 logits of sub-pixel c
+                const int prow = q * 32 + lane;
+                const int rows_valid = (min(m.height, y0 + m.R) - y0) * m.width;
+                const bool valid = prow < rows_valid;
+                const int pix = y0 * m.width + prow;
+                const int t = pix * m.in_ch + c;
+                const size_t at = (size_t)n * m.T + t;
+                const float *bias = m.bias[m.n_conv] + (size_t)c * 256;
+                float best = -INFINITY;
+                int bi = 0;
+                for (int c0 = 0; c0 < 256; c0 += 32) {
+                    float v[32];
+                    tmem_ld32(tbase + (uint32_t)c0, v);
+                    if (!valid) continue;
+                    if (kind == EPI_LOGITS) {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) zout[at * 256 + c0 + i] = v[i] + bias[c0 + i];
+                    } else {
+                        const float *gg = r.noise + at * 256 + c0;
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4) {
+                            const float4 b4 = __ldg(reinterpret_cast<const float4 *>(bias + c0 + i));
+                            const float4 g4 = __ldg(reinterpret_cast<const float4 *>(gg + i));
+                            const float s0 = (v[i] + b4.x) + g4.x, s1 = (v[i + 1] + b4.y) + g4.y;
+                            const float s2 = (v[i + 2] + b4.z) + g4.z, s3 = (v[i + 3] + b4.w) + g4.w;
+                            if (s0 > best) { best = s0; bi = c0 + i; }
+                            if (s1 > best) { best = s1; bi = c0 + i + 1; }
+                            if (s2 > best) { best = s2; bi = c0 + i + 2; }
+                            if (s3 > best) { best = s3; bi = c0 + i + 3; }
+                        }
+                    }
+                }
+                if (kind == EPI_CAT && valid && t >= w.plo && t < w.phi) {
+                    if ((int)r.x[at] != bi) {
+                        r.x[at] = (uint8_t)bi;
+                        ((__nv_bfloat16 *)m.act[0])[((size_t)n * m.height * m.width + pix) * 64 + c] =
+                            __float2bfloat16_rn(m.lut[bi]);
+                        if (flag) {
+                            r.smp_changed[parity * r.batch + n] = 1;
+                            any_changed = true;
+                            first = min(first, t);
+                        }
+                    }
+                }
+                release_acc();
+            }
+            advance_acc();
+        }
+        if (flag) {
+            const bool wany = __any_sync(0xffffffffu, any_changed);
+            if (wany) {
+                const int wmin = __reduce_min_sync(0xffffffffu, first);
+                if (lane == 0) {
+                    atomicMin(&r.ctl->agg_minfirst[parity], wmin);
+                    atomicOr(&r.ctl->agg_any[parity], 1);
+                }
+            }
+        }
+    }
+
+    __device__ bool layer_phase(int l, int kind, const Win &w, bool flag, int parity, float *zout)
+    {
+        const bool head = (l == m.n_conv);
+        int yt_lo, yt_hi;
+        live_rows(head, w, yt_lo, yt_hi);
+        const int nyl = yt_hi - yt_lo;
+        const int ntiles = sh.n_img * nyl * (head ? m.in_ch : 1);
+        if (threadIdx.x == 0) {
+            for (int id = blockIdx.x; id < ntiles; id += gridDim.x) issued++;
+            if (blockIdx.x == 0) skipped += (unsigned long long)(r.batch * m.nyt - sh.n_img * nyl) * (head ? m.in_ch : 1);
+        }
+        if (ntiles == 0) return false;
+        if (warp == 0) {
+            if (lane == 0) producer(l, yt_lo, nyl, ntiles);
+        } else if (warp == 1) {
+            if (lane == 0) mma_issuer(l, ntiles);
+        } else {
+            epilogue(l, kind, w, flag, parity, zout, yt_lo, nyl, ntiles);
+        }
+        return true;
+    }
+
+    __device__ bool forward_logits(float *zout)
+    {
+        const Win w = make_win(0, m.T, 0, m.T);
+        for (int l = 0; l < m.n_conv; ++l) {
+            layer_phase(l, EPI_HIDDEN, w, false, 0, nullptr);
+            if (!barrier()) return false;
+        }
+        layer_phase(m.n_conv, EPI_LOGITS, w, false, 0, zout);
+        return barrier();
+    }
+
+    __device__ bool step(const Win &w, bool flag, int parity)
+    {
+        for (int l = 0; l < m.n_conv; ++l)
+            if (layer_phase(l, EPI_HIDDEN, w, false, 0, nullptr))
+                if (!barrier()) return false;
+        layer_phase(m.n_conv, EPI_CAT, w, flag, parity, nullptr);
+        return barrier();
+    }
+};
+
+__global__ void __launch_bounds__(NTH, 1)
+conv_tc_kernel(const __grid_constant__ ConvDev m, const __grid_constant__ RunArgs r)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ ConvShared sh;
+    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < N_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 4); }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+    }
+    if (warp == 1) tmem_alloc(&sh.tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    ConvEngine e(m, r, sh, ring);
+    e.tmem_base = sh.tmem_base;
+    DriverResult res = made_driver(e, m.T, r);
+    if (e.dead) res.alive = false;
+
+    tc_fence_before();
+    __syncthreads();
+    if (!res.alive || ld_volatile_i32(&r.ctl->abort) != 0) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);      // let copies still in flight land
+        res.alive = false;
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(e.tmem_base, 512);
+    }
+    driver_finish(r, res, e.issued, e.skipped);
+}
+
+}  // namespace
+
+// --------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn conv_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+        return nullptr;
+    fn = (EncodeTiledFn)p;
+    return fn;
+}
+
+static bool encode_nd(CUtensorMap *out, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides,
+                      const cuuint32_t *box)
+{
+    EncodeTiledFn fn = conv_encode_fn();
+    if (!fn) return false;
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <typename T>
+static bool upload(js_model *mo, const T *host, size_t count, T **dev)
+{
+    void *p = nullptr;
+    if (cudaMalloc(&p, std::max<size_t>(count * sizeof(T), 16)) != cudaSuccess) return false;
+    mo->allocs.push_back(p);
+    if (host) {
+        if (cudaMemcpy(p, host, count * sizeof(T), cudaMemcpyHostToDevice) != cudaSuccess) return false;
+    } else if (cudaMemset(p, 0, count * sizeof(T)) != cudaSuccess) {
+        return false;
+    }
+    *dev = (T *)p;
+    return true;
+}
+
+// Builds the device model of a masked-conv stack.  JS_OK, JS_ERR_UNSUPPORTED for shapes the
+// kernel does not cover, JS_ERR_CUDA on runtime failures.
+int js_conv_build(js_model *mo, const js_conv_desc *d)
+{
+    ConvDev &v = mo->conv;
+    if (d->prec != JS_BF16 || d->C != 256 || d->n_lut != 256) return JS_ERR_UNSUPPORTED;
+    if (d->in_ch < 1 || d->in_ch > 8 || (d->ch != 64 && d->ch != 128)) return JS_ERR_UNSUPPORTED;
+    if (d->width < 8 || d->width > 128 || (128 % d->width) != 0 || d->height < 1) return JS_ERR_UNSUPPORTED;
+    if (d->n_conv < 1 || d->n_conv > JS_MAXL || d->max_batch > MAX_IMAGES) return JS_ERR_UNSUPPORTED;
+    if (!conv_encode_fn()) return JS_ERR_UNSUPPORTED;
+    v.height = d->height; v.width = d->width; v.in_ch = d->in_ch; v.ch = d->ch; v.n_conv = d->n_conv; v.C = d->C;
+    v.T = d->height * d->width * d->in_ch;
+    v.R = 128 / d->width;
+    v.nyt = (d->height + v.R - 1) / v.R;
+    const int ch = d->ch, nb = mo->max_batch;
+    const size_t npix = (size_t)nb * d->height * d->width;
+    auto group = [&](int k) { return (int)(((long long)d->in_ch * k) / ch); };
+
+    std::vector<CUtensorMap> mapsA(d->n_conv + 1), mapsW(d->n_conv + 1);
+    for (int l = 0; l <= d->n_conv; ++l) {
+        const int c_l = l == 0 ? 64 : ch;                 // channels of act[l] (the image is padded to 64)
+        if (l < d->n_conv) v.cin_pad[l] = c_l;
+        __nv_bfloat16 *a = nullptr;
+        if (!upload<__nv_bfloat16>(mo, nullptr, npix * c_l, &a)) return JS_ERR_CUDA;
+        v.act[l] = a;
+        const cuuint64_t dims[4] = {(cuuint64_t)c_l, (cuuint64_t)d->width, (cuuint64_t)d->height, (cuuint64_t)nb};
+        const cuuint64_t strides[3] = {(cuuint64_t)c_l * 2, (cuuint64_t)d->width * c_l * 2,
+                                       (cuuint64_t)d->height * d->width * c_l * 2};
+        const cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)d->width, (cuuint32_t)v.R, 1};
+        if (!encode_nd(&mapsA[l], a, 4, dims, strides, box)) return JS_ERR_UNSUPPORTED;
+    }
+    static const int tky[5] = {0, 0, 0, 1, 1}, tkx[5] = {0, 1, 2, 0, 1};
+    for (int l = 0; l < d->n_conv; ++l) {
+        const int cin = l == 0 ? d->in_ch : ch, cpad = v.cin_pad[l];
+        std::vector<__nv_bfloat16> wp((size_t)5 * ch * cpad, __float2bfloat16_rn(0.0f));
+        for (int tap = 0; tap < 5; ++tap)
+            for (int co = 0; co < ch; ++co)
+                for (int ci = 0; ci < cin; ++ci) {
+                    bool keep = true;
+                    if (tap == 4) {                       // centre tap: colour-group mask, type A then type B
+                        const int gi = l == 0 ? ci : group(ci), go = group(co);
+                        keep = l == 0 ? (gi < go) : (gi <= go);
+                    }
+                    const float w = keep ? d->W[l][(((size_t)co * 3 + tky[tap]) * 3 + tkx[tap]) * cin + ci] : 0.0f;
+                    wp[((size_t)tap * ch + co) * cpad + ci] = __float2bfloat16_rn(w);
+                }
+        __nv_bfloat16 *wd = nullptr;
+        if (!upload<__nv_bfloat16>(mo, wp.data(), wp.size(), &wd)) return JS_ERR_CUDA;
+        const cuuint64_t dims[2] = {(cuuint64_t)cpad, (cuuint64_t)5 * ch};
+        const cuuint64_t strides[1] = {(cuuint64_t)cpad * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)ch};
+        if (!encode_nd(&mapsW[l], wd, 2, dims, strides, box)) return JS_ERR_UNSUPPORTED;
+        float *bd = nullptr;
+        if (!upload<float>(mo, d->b[l], ch, &bd)) return JS_ERR_CUDA;
+        v.bias[l] = bd;
+    }
+    {
+        const int nout = d->in_ch * d->C;
+        std::vector<__nv_bfloat16> wh((size_t)nout * ch);
+        for (int o = 0; o < nout; ++o)
+            for (int ci = 0; ci < ch; ++ci)
+                wh[(size_t)o * ch + ci] =
+                    __float2bfloat16_rn(group(ci) <= o / d->C ? d->W[d->n_conv][(size_t)o * ch + ci] : 0.0f);
+        __nv_bfloat16 *wd = nullptr;
+        if (!upload<__nv_bfloat16>(mo, wh.data(), wh.size(), &wd)) return JS_ERR_CUDA;
+        const cuuint64_t dims[2] = {(cuuint64_t)ch, (cuuint64_t)nout};
+        const cuuint64_t strides[1] = {(cuuint64_t)ch * 2};
+        const cuuint32_t box[2] = {(cuuint32_t)BK, 256};
+        if (!encode_nd(&mapsW[d->n_conv], wd, 2, dims, strides, box)) return JS_ERR_UNSUPPORTED;
+        float *bd = nullptr;
+        if (!upload<float>(mo, d->b[d->n_conv], nout, &bd)) return JS_ERR_CUDA;
+        v.bias[d->n_conv] = bd;
+    }
+    {
+        std::vector<float> lut(d->lut, d->lut + d->n_lut);
+        for (auto &f : lut) f = __bfloat162float(__float2bfloat16_rn(f));
+        float *ld = nullptr;
+        if (!upload<float>(mo, lut.data(), lut.size(), &ld)) return JS_ERR_CUDA;
+        v.lut = ld;
+    }
+    CUtensorMap *pa = nullptr, *pw = nullptr;
+    if (!upload<CUtensorMap>(mo, mapsA.data(), mapsA.size(), &pa)) return JS_ERR_CUDA;
+    if (!upload<CUtensorMap>(mo, mapsW.data(), mapsW.size(), &pw)) return JS_ERR_CUDA;
+    v.tmAct = pa;
+    v.tmW = pw;
+    if (cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES) != cudaSuccess) {
+        cudaGetLastError();
+        return JS_ERR_UNSUPPORTED;
+    }
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    mo->conv_max_grid = sms;
+    mo->conv_T = v.T;
+    mo->conv_C = v.C;
+    return JS_OK;
+}
+
+int js_launch_conv_tc(const js_model *mo, const RunArgs &r, cudaStream_t stream)
+{
+    const ConvDev &v = mo->conv;
+    const int tiles = r.batch * v.nyt * v.in_ch;
+    const int grid = std::max(1, std::min(mo->conv_max_grid, tiles));
+    void *args[2] = {(void *)&v, (void *)&r};
+    cudaError_t e = cudaLaunchCooperativeKernel((const void *)conv_tc_kernel, dim3(grid), dim3(NTH), args, SMEM_BYTES,
+                                                stream);
+    return e == cudaSuccess ? 0 : (int)e;
+}

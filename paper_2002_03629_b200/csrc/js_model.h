@@ -22,6 +22,19 @@ struct TcDev {
     int stage_bytes, n_stages, smem_bytes;
 };
 
+// Device view of a masked-convolution stack (tensor-core kernel only).
+struct ConvDev {
+    int height, width, in_ch, ch, n_conv, C, T;
+    int R;                              // image rows per 128-pixel tile
+    int nyt;                            // row tiles per image
+    int cin_pad[JS_MAXL];               // input channels of conv layer l, padded to a multiple of 64
+    void *act[JS_MAXL + 1];             // NHWC bf16; act[0] = encoded image padded to 64 channels
+    const float *bias[JS_MAXL + 1];     // conv biases, head bias at [n_conv]
+    const float *lut;
+    const CUtensorMap *tmAct;           // [n_conv+1] 4-D maps {channel, x, y, image}, box 64 x width x R x 1
+    const CUtensorMap *tmW;             // [n_conv+1] 2-D maps of the packed weights
+};
+
 struct js_model {
     int kind = 0;                 // 0 masked MLP, 1 masked-conv stack
     int max_batch = 0;
@@ -38,8 +51,12 @@ struct js_model {
     int max_grid_generic = 0;
     TcDev tc{};
     int tc_ok = 0, tc_max_grid = 0;
+    ConvDev conv{};
+    int conv_max_grid = 0;
     js_stats stats{};
 };
 
 int js_tc_prepare(js_model *m);
 int js_launch_made_tc(const js_model *m, const RunArgs &r, cudaStream_t stream);
+int js_conv_build(js_model *m, const js_conv_desc *d);
+int js_launch_conv_tc(const js_model *m, const RunArgs &r, cudaStream_t stream);

@@ -69,11 +69,10 @@ struct DriverResult {
 };
 
 template <class E>
-__device__ DriverResult made_driver(E &e, const MadeDev &m, const RunArgs &r)
+__device__ DriverResult made_driver(E &e, int T_, const RunArgs &r)
 {
     DriverResult res = {JS_OK, 0, 0, true};
     JsCtl *ctl = r.ctl;
-    const int T_ = m.T;
 
     if (r.kmode == KM_FORWARD) {
         e.init(r.x_in);

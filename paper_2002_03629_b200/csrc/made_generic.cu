@@ -406,7 +406,7 @@ __global__ void __launch_bounds__(NTHREADS) made_generic_kernel(const __grid_con
 {
     __shared__ Smem s;
     GenericEngine<T> e(s, m, r);
-    const DriverResult res = made_driver(e, m, r);
+    const DriverResult res = made_driver(e, m.T, r);
     driver_finish(r, res, e.issued, e.skipped);
 }
 

@@ -1,0 +1,155 @@
+"""Parity of the CUDA masked-convolution sampler with the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from parity import check_samples, logits_close
+
+pytestmark = pytest.mark.gpu
+
+# two row tiles per image, the second one ragged (12 rows, 8 rows per 128-pixel tile)
+SMALL = si.ConvConfig("conv_small", 61, height=12, width=16, in_ch=3, ch=64, layers=3, C=256, batch=3)
+_cache = {}
+
+
+def pkg():
+    import __graft_entry__ as ge
+    ge.build()
+    import paper_2002_03629_b200 as p
+    return p
+
+
+class ConvCase:
+    def __init__(self, cfg, gain=1.0, threads=8):
+        p = pkg()
+        self.p, self.cfg = p, cfg
+        W, b = si.conv_weights(cfg)
+        self.W = [w * np.float32(gain) for w in W]
+        self.b = b
+        self.lut = si.conv_lut(cfg)
+        self.noise = si.draw_noise(cfg)
+        self.nk = cfg.noise_kind
+        self.orc = oracle.from_config(cfg, self.W, self.b, self.lut)
+        self.model = p.Model.from_config(cfg, self.W, self.b, self.lut)
+        self.d_noise = torch.from_numpy(self.noise).cuda()
+        self.xstar = self.orc.sequential_batch(self.noise, self.nk, threads=threads)
+
+    def run(self, mode, block=0, max_iters=0, init=None):
+        cfg, p = self.cfg, self.p
+        out = torch.full((cfg.batch, cfg.D), 255, dtype=torch.uint8, device="cuda")
+        iters = torch.full((cfg.batch,), -1, dtype=torch.int32, device="cuda")
+        d_init = None if init is None else torch.from_numpy(init).cuda()
+        rc = p.jacobi_sample(self.model, self.d_noise, self.nk, d_init, mode, block, max_iters, out, iters)
+        return rc, out.cpu().numpy(), iters.cpu().numpy()
+
+
+def small():
+    if "s" not in _cache:
+        _cache["s"] = ConvCase(SMALL, gain=2.0)
+    return _cache["s"]
+
+
+def test_conv_logits_match_oracle():
+    c = small()
+    cfg, p = c.cfg, c.p
+    x = si.random_init(cfg, salt=5)
+    logits = torch.empty((cfg.batch, cfg.D, cfg.C), dtype=torch.float32, device="cuda")
+    assert p.js_forward_logits(c.model, torch.from_numpy(x).cuda(), logits) == 0
+    got = logits.cpu().numpy()
+    ref = np.stack([c.orc.forward_logits(x[s]) for s in range(cfg.batch)])
+    err, ok = logits_close(got, ref, 2e-2)
+    assert ok, err
+
+
+@pytest.mark.parametrize("skip,compact", [(1, 1), (0, 1), (1, 0)])
+def test_conv_jacobi_matches_sequential_and_counts(skip, compact):
+    c = small()
+    p, cfg = c.p, c.cfg
+    c.model.set_option(p.JS_OPT_FRONTIER_SKIP, skip)
+    c.model.set_option(p.JS_OPT_COMPACT, compact)
+    try:
+        for init in (None, si.random_init(cfg, salt=1)):
+            rc, x, it = c.run(p.JS_JACOBI, init=init)
+            assert rc == 0
+            audit = check_samples(c.orc, x, c.xstar, c.noise, c.nk)
+            ref = [c.orc.jacobi(c.noise[s], c.nk, None if init is None else init[s])[1] for s in range(cfg.batch)]
+            clean = [s for s in range(cfg.batch) if s not in audit["excused_samples"]]
+            np.testing.assert_array_equal(it[clean], np.array(ref)[clean])
+            assert max(ref) > 3, "the small conv case should need more than a few iterations"
+    finally:
+        c.model.set_option(p.JS_OPT_FRONTIER_SKIP, 1)
+        c.model.set_option(p.JS_OPT_COMPACT, 1)
+
+
+@pytest.mark.parametrize("seq_skip", [0, 1])
+def test_conv_sequential_and_gauss_seidel(seq_skip):
+    c = small()
+    p, cfg = c.p, c.cfg
+    c.model.set_option(p.JS_OPT_SEQ_SKIP, seq_skip)
+    try:
+        out = torch.empty((cfg.batch, cfg.D), dtype=torch.uint8, device="cuda")
+        assert p.sequential_sample(c.model, c.d_noise, c.nk, out) == 0
+        check_samples(c.orc, out.cpu().numpy(), c.xstar, c.noise, c.nk)
+        rc, x, it = c.run(p.JS_GAUSS_SEIDEL, init=si.random_init(cfg, salt=2))
+        assert rc == 0 and np.all(it == 1)
+        check_samples(c.orc, x, c.xstar, c.noise, c.nk)
+    finally:
+        c.model.set_option(p.JS_OPT_SEQ_SKIP, 0)
+
+
+@pytest.mark.parametrize("B", [48, 100, 576])
+def test_conv_gs_jacobi(B):
+    c = small()
+    p, cfg = c.p, c.cfg
+    for init in (None, si.random_init(cfg, salt=3)):
+        rc, x, it = c.run(p.JS_GS_JACOBI, block=B, init=init)
+        assert rc == 0
+        audit = check_samples(c.orc, x, c.xstar, c.noise, c.nk)
+        ref = [c.orc.gs_jacobi(c.noise[s], c.nk, B, None if init is None else init[s])[1] for s in range(cfg.batch)]
+        clean = [s for s in range(cfg.batch) if s not in audit["excused_samples"]]
+        np.testing.assert_array_equal(it[clean], np.array(ref)[clean])
+
+
+def test_conv_max_iters_and_unsupported_mode():
+    c = small()
+    p, cfg = c.p, c.cfg
+    rc, x, it = c.run(p.JS_JACOBI, max_iters=2)
+    assert rc == p.JS_NOT_CONVERGED and np.all(it == 2)
+    ref = np.stack([c.orc.jacobi(c.noise[s], c.nk, None, 2)[0] for s in range(cfg.batch)])
+    assert np.mean(x == ref) > 0.999
+    with pytest.raises(p.JsError) as e:
+        c.run(p.JS_JACOBI_GS, block=48)
+    assert e.value.code == p.JS_ERR_UNSUPPORTED
+
+
+def test_conv_full_size_config():
+    """32x32x3, eight masked 3x3 layers of 128 channels, batch 16: every image against the
+    oracle's feedforward pass; Jacobi, banded sequential order and GS-Jacobi with two-row blocks."""
+    cfg = si.CONFIGS["conv_32"]
+    c = ConvCase(cfg, threads=16)
+    p = c.p
+    rc, x, it = c.run(p.JS_JACOBI)
+    assert rc == 0
+    audit = check_samples(c.orc, x, c.xstar, c.noise, c.nk)
+    print(f"conv_32: jacobi iters mean {it.mean():.2f} max {it.max()} excused {audit}")
+    assert it.max() <= cfg.D
+    c.model.set_option(p.JS_OPT_SEQ_SKIP, 1)
+    out = torch.empty((cfg.batch, cfg.D), dtype=torch.uint8, device="cuda")
+    assert p.sequential_sample(c.model, c.d_noise, c.nk, out) == 0
+    c.model.set_option(p.JS_OPT_SEQ_SKIP, 0)
+    check_samples(c.orc, out.cpu().numpy(), c.xstar, c.noise, c.nk)
+    rc, x, it2 = c.run(p.JS_GS_JACOBI, block=2 * cfg.width * cfg.in_ch)
+    assert rc == 0
+    check_samples(c.orc, x, c.xstar, c.noise, c.nk)
+    print(f"conv_32: gs-jacobi (2 rows) inner iterations mean {it2.mean():.1f}")
+    # logits of two images
+    xi = si.random_init(cfg, salt=9)
+    logits = torch.empty((cfg.batch, cfg.D, cfg.C), dtype=torch.float32, device="cuda")
+    assert p.js_forward_logits(c.model, torch.from_numpy(xi).cuda(), logits) == 0
+    rows = [0, cfg.batch - 1]
+    ref = np.stack(c.orc.map_batch(lambda i: c.orc.forward_logits(xi[rows[i]]), 2, threads=2))
+    err, ok = logits_close(logits[rows].cpu().numpy(), ref, 2e-2)
+    print(f"conv_32: max relative logit error {err:.3e}")
+    assert ok, err
