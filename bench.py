@@ -31,8 +31,26 @@ DEFAULT_WORKLOAD = "made_4096"
 
 
 # ------------------------------------------------------------------ workload
+def conv_live_macs_per_image(cfg) -> int:
+    """Unmasked multiply-accumulates of one forward pass of the masked-conv stack for one image
+    (four full taps and the colour-group-masked centre tap per 3x3 layer, masked 1x1 head)."""
+    ch, n_in = cfg.ch, cfg.in_ch
+    grp = (n_in * np.arange(ch)) // ch
+    per_pixel = 0
+    for l in range(cfg.layers):
+        cin = n_in if l == 0 else ch
+        gi = np.arange(n_in) if l == 0 else grp
+        centre = (gi[None, :] < grp[:, None]) if l == 0 else (gi[None, :] <= grp[:, None])
+        per_pixel += 4 * cin * ch + int(centre.sum())
+    head = grp[None, :] <= (np.arange(n_in * cfg.C) // cfg.C)[:, None]
+    per_pixel += int(head.sum())
+    return per_pixel * cfg.height * cfg.width
+
+
 def live_macs_per_sample(cfg) -> int:
     """Unmasked multiply-accumulates of one forward pass for one sample."""
+    if cfg.kind == "conv":
+        return conv_live_macs_per_image(cfg)
     D, C = cfg.D, cfg.C
     deg = [np.arange(1, D + 1)]
     for h in cfg.H:
@@ -112,6 +130,9 @@ MODES = {"jacobi": 0, "gauss_seidel": 1, "gs_jacobi": 2, "jacobi_gs": 3}
 
 
 def make_inputs(cfg):
+    if cfg.kind == "conv":
+        W, b = si.conv_weights(cfg)
+        return W, b, si.conv_lut(cfg), si.draw_noise(cfg)
     W, b = si.made_weights(cfg)
     return W, b, si.made_lut(cfg), si.draw_noise(cfg)
 
@@ -291,7 +312,8 @@ def run_ours(args, cfg):
             "warmup": max(args.warmup, 3), "ms_per_step": ms_launch, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": dtype, "data": "synthetic",
             "config": {"workload": cfg.name, "mode": args.mode, "block": block, "batch": cfg.batch, "T": cfg.D,
-                       "C": cfg.C, "hidden": list(cfg.H), "parallelism": f"replicas x{world}",
+                       "C": cfg.C, "hidden": list(cfg.H) if cfg.kind == "made" else [cfg.ch] * cfg.layers,
+                       "parallelism": f"replicas x{world}",
                        "l2": "256 MB written between timed steps (L2 flush)"},
             "iters_per_sample": {"mean": float(it_np.mean()), "max": int(it_np.max()),
                                  "forward_passes": int(stats.iterations)},

@@ -130,26 +130,46 @@ def test_conv_full_size_config():
     cfg = si.CONFIGS["conv_32"]
     c = ConvCase(cfg, threads=16)
     p = c.p
+    # teacher-forced logits of three images: relative tolerance, and E for the tie margin
+    xi = si.random_init(cfg, salt=9)
+    logits = torch.empty((cfg.batch, cfg.D, cfg.C), dtype=torch.float32, device="cuda")
+    assert p.js_forward_logits(c.model, torch.from_numpy(xi).cuda(), logits) == 0
+    rows = [0, 5, cfg.batch - 1]
+    ref = np.stack(c.orc.map_batch(lambda i: c.orc.forward_logits(xi[rows[i]]), 3, threads=3))
+    got = logits[rows].cpu().numpy()
+    # 2e-2 is the tolerance for networks of up to four bf16-rounded hidden layers; rounding
+    # differences compound with every further rounded layer, so it is scaled by layers / 4
+    tol = 2e-2 * max(1.0, cfg.layers / 4.0)
+    err, ok = logits_close(got, ref, tol)
+    frac_within = float(np.mean(np.abs(got - ref) <= 2e-2 * np.maximum(np.abs(ref), np.sqrt(np.mean(ref ** 2)))))
+    print(f"conv_32: share of logits within 2e-2: {frac_within:.6f}")
+    assert frac_within > 0.9999
+    E = float(np.abs(got - ref).max())
+    margin = max(1e-3, 2 * E)
+    print(f"conv_32: max relative logit error {err:.3e}, max absolute {E:.3e} -> tie margin {margin:.3e}")
+    assert ok, err
+    assert margin < 0.05, "eight bf16 layers should not move a logit by more than a few 1e-2"
+
     rc, x, it = c.run(p.JS_JACOBI)
     assert rc == 0
-    audit = check_samples(c.orc, x, c.xstar, c.noise, c.nk)
-    print(f"conv_32: jacobi iters mean {it.mean():.2f} max {it.max()} excused {audit}")
+    audit = check_samples(c.orc, x, c.xstar, c.noise, c.nk, margin=margin)
+    strict = sum(1 for s in range(cfg.batch) if not np.array_equal(x[s], c.xstar[s]))
+    print(f"conv_32: jacobi iters mean {it.mean():.2f} max {it.max()}; samples differing from the oracle: "
+          f"{strict}/{cfg.batch}, all from near-ties: {audit}")
     assert it.max() <= cfg.D
+    # iteration counts against the oracle's, on the images that match it bit for bit
+    clean = [s for s in range(cfg.batch) if s not in audit["excused_samples"]]
+    ref_it = c.orc.map_batch(lambda i: c.orc.jacobi(c.noise[clean[i]], c.nk)[1], len(clean), threads=16)
+    np.testing.assert_array_equal(it[clean], np.array(ref_it))
     c.model.set_option(p.JS_OPT_SEQ_SKIP, 1)
     out = torch.empty((cfg.batch, cfg.D), dtype=torch.uint8, device="cuda")
     assert p.sequential_sample(c.model, c.d_noise, c.nk, out) == 0
     c.model.set_option(p.JS_OPT_SEQ_SKIP, 0)
-    check_samples(c.orc, out.cpu().numpy(), c.xstar, c.noise, c.nk)
-    rc, x, it2 = c.run(p.JS_GS_JACOBI, block=2 * cfg.width * cfg.in_ch)
+    seq = out.cpu().numpy()
+    check_samples(c.orc, seq, c.xstar, c.noise, c.nk, margin=margin)
+    # on the device every solver must reach the very same fixed point, bit for bit
+    np.testing.assert_array_equal(seq, x)
+    rc, x2, it2 = c.run(p.JS_GS_JACOBI, block=2 * cfg.width * cfg.in_ch)
     assert rc == 0
-    check_samples(c.orc, x, c.xstar, c.noise, c.nk)
+    np.testing.assert_array_equal(x2, x)
     print(f"conv_32: gs-jacobi (2 rows) inner iterations mean {it2.mean():.1f}")
-    # logits of two images
-    xi = si.random_init(cfg, salt=9)
-    logits = torch.empty((cfg.batch, cfg.D, cfg.C), dtype=torch.float32, device="cuda")
-    assert p.js_forward_logits(c.model, torch.from_numpy(xi).cuda(), logits) == 0
-    rows = [0, cfg.batch - 1]
-    ref = np.stack(c.orc.map_batch(lambda i: c.orc.forward_logits(xi[rows[i]]), 2, threads=2))
-    err, ok = logits_close(logits[rows].cpu().numpy(), ref, 2e-2)
-    print(f"conv_32: max relative logit error {err:.3e}")
-    assert ok, err
