@@ -153,9 +153,10 @@ typedef struct {
 int js_get_stats(const js_model *m, js_stats *out);
 
 /* Device-side timeline of the most recent call made with JS_OPT_TRACE on (tensor-core kernels):
- * globaltimer nanoseconds, layout [2][256][8] = [first CTA, last CTA][phase][slot]; a phase is one
+ * globaltimer nanoseconds, layout [2][256][12] = [first CTA, last CTA][phase][slot]; a phase is one
  * layer of one forward pass; slots: 0 phase start, 1 first operands landed, 2 last MMA issued,
- * 3 accumulator complete, 4 epilogue stored, 5 left the grid barrier; 0 = not recorded.
+ * 3 accumulator complete, 4 epilogue stored, 5 left the grid barrier, 6-11 points inside the
+ * epilogue; 0 = not recorded.
  * Copies at most `capacity` values to the HOST array `out`, returns how many. */
 int js_get_trace(const js_model *m, unsigned long long *out, int capacity);
 

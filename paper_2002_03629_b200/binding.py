@@ -183,8 +183,8 @@ class Model:
         return s
 
     def trace(self) -> np.ndarray:
-        """js_get_trace: device timestamps [2 CTAs][256 phases][8 slots] of the last traced call."""
-        buf = np.zeros((2, 256, 8), dtype=np.uint64)
+        """js_get_trace: device timestamps [2 CTAs][256 phases][12 slots] of the last traced call."""
+        buf = np.zeros((2, 256, 12), dtype=np.uint64)
         _check(load_library().js_get_trace(self._h, buf.ctypes.data_as(C.c_void_p), buf.size), "js_get_trace")
         return buf
 

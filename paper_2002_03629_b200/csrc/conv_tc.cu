@@ -325,7 +325,8 @@ struct ConvEngine {
                         ((__nv_bfloat16 *)m.act[0])[((size_t)n * m.height * m.width + pix) * 64 + c] =
                             __float2bfloat16_rn(m.lut[bi]);
                         if (flag) {
-                            r.smp_changed[parity * r.batch + n] = 1;
+                            int *f = &r.smp_changed[parity * r.batch + n];     // look first: stores to one
+                            if (ld_volatile_i32(f) == 0) *f = 1;                 // address serialise in L2
                             any_changed = true;
                             first = min(first, t);
                         }
@@ -369,24 +370,15 @@ struct ConvEngine {
         return true;
     }
 
-    __device__ bool forward_logits(float *zout)
+    __device__ bool step(const Win &w, bool flag, int parity, float *zout)
     {
-        const Win w = make_win(0, m.T, 0, m.T);
-        for (int l = 0; l < m.n_conv; ++l) {
-            layer_phase(l, EPI_HIDDEN, w, false, 0, nullptr);
-            if (!barrier()) return false;
-        }
-        layer_phase(m.n_conv, EPI_LOGITS, w, false, 0, zout);
-        return barrier();
-    }
-
-    __device__ bool step(const Win &w, bool flag, int parity)
-    {
-        for (int l = 0; l < m.n_conv; ++l)
-            if (layer_phase(l, EPI_HIDDEN, w, false, 0, nullptr))
+        for (int l = 0; l <= m.n_conv; ++l) {
+            const bool last = (l == m.n_conv);
+            const bool did = layer_phase(l, last ? (zout ? EPI_LOGITS : EPI_CAT) : EPI_HIDDEN, w, last && flag, parity, zout);
+            if (did || last)
                 if (!barrier()) return false;
-        layer_phase(m.n_conv, EPI_CAT, w, flag, parity, nullptr);
-        return barrier();
+        }
+        return true;
     }
 };
 

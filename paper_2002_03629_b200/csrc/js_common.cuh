@@ -10,7 +10,7 @@
 
 #define JS_MAXL 8
 #define JS_TRACE_PHASES 256
-#define JS_TRACE_SLOTS 8
+#define JS_TRACE_SLOTS 12
 #define JS_GT 64          // output-tile edge of the CUDA-core GEMM phases
 
 enum { KM_JACOBI = 0, KM_SEQ = 1, KM_GS_JACOBI = 2, KM_JACOBI_GS = 3, KM_FORWARD = 4 };

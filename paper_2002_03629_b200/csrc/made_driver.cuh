@@ -68,105 +68,19 @@ struct DriverResult {
     bool alive;
 };
 
+// The solver loops are written as ONE loop with ONE call of the engine's forward pass: the
+// engines inline their whole pipeline into that call, and a copy per solver would multiply the
+// kernel's code size (the persistent kernels are instruction-cache sensitive).
 template <class E>
 __device__ DriverResult made_driver(E &e, int T_, const RunArgs &r)
 {
     DriverResult res = {JS_OK, 0, 0, true};
     JsCtl *ctl = r.ctl;
+    const int mode = r.kmode;
 
-    if (r.kmode == KM_FORWARD) {
-        e.init(r.x_in);
+    if (mode == KM_JACOBI_GS) {
+        e.init(r.init);
         if (!e.barrier()) { res.alive = false; return res; }
-        if (!e.forward_logits(r.logits_out)) { res.alive = false; return res; }
-        res.iterations = 1;
-        return res;
-    }
-
-    e.init(r.kmode == KM_SEQ ? (const uint8_t *)nullptr : r.init);
-    if (!e.barrier()) { res.alive = false; return res; }
-
-    if (r.kmode == KM_SEQ) {
-        // Eq. 1 in strict order: step t keeps position t of a forward pass.
-        for (int t = 0; t < T_; ++t) {
-            Win w = make_win(0, T_, t, t + 1);
-            if (r.seq_skip) w.hdeg_lo = t - 1, w.hdeg_hi = t;     // only the units that became computable
-            else w.olo = 0, w.ohi = T_;                           // the whole network, every step
-            if (!e.step(w, false, 0)) { res.alive = false; return res; }
-            res.iterations++;
-        }
-        res.frontier = T_;
-        if (blockIdx.x == 0 && r.out_iters)
-            for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.out_iters[b] = 1;
-        return res;
-    }
-
-    if (r.kmode == KM_JACOBI) {
-        // Algorithm 1 with per-sample stopping.
-        const int cap = (r.max_iters > 0 && r.max_iters < T_) ? r.max_iters : T_;
-        int fin_x = 0, fin_h = 0;
-        for (int k = 1;; ++k) {
-            const int p = k & 1;
-            const Win w = r.frontier_skip ? make_win(fin_h, T_, fin_x, T_) : make_win(0, T_, 0, T_);
-            if (!e.step(w, true, p)) { res.alive = false; return res; }
-            res.iterations++;
-            const int any = ld_volatile_i32(&ctl->agg_any[p]);
-            const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
-            book_samples(r, p, k, k == cap, false, true);
-            reset_other_parity(r, p);
-            fin_h = max(fin_h, fin_x);
-            fin_x = any ? max(fin_x + 1, min(mf + 1, T_)) : T_;
-            if (!any || k == cap) {
-                if (any && cap < T_) res.status = JS_NOT_CONVERGED;
-                break;
-            }
-            // samples that stopped changing are at their fixed point: drop them from the working
-            // batch when that frees a whole tile of rows (hidden rows are then recomputed)
-            if (r.compact) {
-                const int c = e.compact(p);
-                if (c < 0) { res.alive = false; return res; }
-                if (c > 0) fin_h = 0;
-            }
-        }
-        res.frontier = fin_x;
-        return res;
-    }
-
-    if (r.kmode == KM_GS_JACOBI) {
-        // Algorithm 3: blocks in order, Jacobi inside the block.
-        const int B = r.block;
-        int fin_x = 0, fin_h = 0, tick = 0;
-        for (int a = 0; a < T_; a += B) {
-            const int bend = min(a + B, T_), len = bend - a;
-            const int cap = (r.max_iters > 0 && r.max_iters < len) ? r.max_iters : len;
-            int lo = a;                         // positions of the block below lo are settled
-            for (int k = 1;; ++k) {
-                const int p = (++tick) & 1;
-                const Win w = r.frontier_skip ? make_win(fin_h, bend - 1, lo, bend) : make_win(0, T_, a, bend);
-                if (!e.step(w, true, p)) { res.alive = false; return res; }
-                res.iterations++;
-                const int any = ld_volatile_i32(&ctl->agg_any[p]);
-                const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
-                book_samples(r, p, k, k == cap, true, false);
-                reset_other_parity(r, p);
-                fin_h = max(fin_h, min(fin_x, bend - 1));
-                lo = any ? max(lo + 1, min(mf + 1, bend)) : bend;
-                fin_x = max(fin_x, lo);
-                if (!any || k == cap) {
-                    if (any && cap < len) res.status = JS_NOT_CONVERGED;
-                    break;
-                }
-            }
-            fin_x = bend;      // positions < bend are never touched again: settled
-            if (blockIdx.x == 0)   // new block: nobody is done (same threads wrote these entries)
-                for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.smp_state[b] = 0;
-        }
-        if (blockIdx.x == 0 && r.out_iters)
-            for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.out_iters[b] = r.smp_state[r.batch + b];
-        res.frontier = T_;
-        return res;
-    }
-
-    if (r.kmode == KM_JACOBI_GS) {
         if constexpr (E::has_jgs) {
             // Algorithm 2: all blocks in parallel, a sequential sweep inside each.
             const int B = r.block, M = (T_ + B - 1) / B;
@@ -196,7 +110,91 @@ __device__ DriverResult made_driver(E &e, int T_, const RunArgs &r)
         }
         return res;
     }
-    res.status = JS_ERR_ARG;
+    if (mode != KM_FORWARD && mode != KM_SEQ && mode != KM_JACOBI && mode != KM_GS_JACOBI) {
+        res.status = JS_ERR_ARG;
+        return res;
+    }
+
+    e.init(mode == KM_FORWARD ? r.x_in : mode == KM_SEQ ? (const uint8_t *)nullptr : r.init);
+    if (!e.barrier()) { res.alive = false; return res; }
+
+    // state shared by the modes
+    const int B = mode == KM_GS_JACOBI ? r.block : T_;     // Jacobi = one block of all positions
+    int fin_x = 0, fin_h = 0;      // see the header comment
+    int a = 0;                     // start of the current block (GS-Jacobi) / position (sequential order)
+    int lo = 0;                    // positions of the current block below lo are settled
+    int k = 0;                     // iteration inside the current block
+    int tick = 0;                  // forward passes with change flags so far (parity of the flag buffers)
+    for (;;) {
+        Win w;
+        bool flag = false;
+        float *zout = nullptr;
+        const int bend = min(a + B, T_), len = bend - a;
+        if (mode == KM_FORWARD) {
+            w = make_win(0, T_, 0, T_);
+            zout = r.logits_out;
+        } else if (mode == KM_SEQ) {
+            // Eq. 1 in strict order: step a keeps position a of a forward pass
+            w = make_win(0, T_, a, a + 1);
+            if (r.seq_skip) w.hdeg_lo = a - 1, w.hdeg_hi = a;     // only the units that became computable
+            else w.olo = 0, w.ohi = T_;                           // the whole network, every step
+        } else {
+            // Algorithm 1 (one block) or the inner loop of Algorithm 3 (block [a, bend))
+            k += 1;
+            tick += 1;
+            flag = true;
+            w = r.frontier_skip ? make_win(fin_h, bend - 1 + (mode == KM_JACOBI), lo, bend)
+                                : make_win(0, T_, a, bend);
+        }
+        const int p = tick & 1;
+        if (!e.step(w, flag, p, zout)) { res.alive = false; return res; }
+        res.iterations++;
+
+        if (mode == KM_FORWARD) break;
+        if (mode == KM_SEQ) {
+            if (++a == T_) break;
+            continue;
+        }
+        const int cap = (r.max_iters > 0 && r.max_iters < len) ? r.max_iters : len;
+        const int any = ld_volatile_i32(&ctl->agg_any[p]);
+        const int mf = ld_volatile_i32(&ctl->agg_minfirst[p]);
+        book_samples(r, p, k, k == cap, mode == KM_GS_JACOBI, mode == KM_JACOBI);
+        reset_other_parity(r, p);
+        fin_h = max(fin_h, min(fin_x, mode == KM_JACOBI ? T_ : bend - 1));
+        lo = any ? max(lo + 1, min(mf + 1, bend)) : bend;
+        fin_x = max(fin_x, lo);
+        if (any && k < cap) {
+            // samples that stopped changing are at their fixed point: drop them from the working
+            // batch when that frees a whole tile of rows (hidden rows are then recomputed)
+            if (mode == KM_JACOBI && r.compact) {
+                const int c = e.compact(p);
+                if (c < 0) { res.alive = false; return res; }
+                if (c > 0) fin_h = 0;
+            }
+            continue;
+        }
+        // the block is finished: unchanged, or at its cap
+        if (any && cap < len) res.status = JS_NOT_CONVERGED;
+        if (mode == KM_JACOBI) break;
+        fin_x = bend;          // positions < bend are never touched again: settled
+        if (blockIdx.x == 0)   // new block: nobody is done (same threads wrote these entries)
+            for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.smp_state[b] = 0;
+        a = bend;
+        lo = a;
+        k = 0;
+        if (a >= T_) break;
+    }
+    if (mode == KM_SEQ) {
+        res.frontier = T_;
+        if (blockIdx.x == 0 && r.out_iters)
+            for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.out_iters[b] = 1;
+    } else if (mode == KM_GS_JACOBI) {
+        res.frontier = T_;
+        if (blockIdx.x == 0 && r.out_iters)
+            for (int b = threadIdx.x; b < r.batch; b += blockDim.x) r.out_iters[b] = r.smp_state[r.batch + b];
+    } else if (mode == KM_JACOBI) {
+        res.frontier = fin_x;
+    }
     return res;
 }
 

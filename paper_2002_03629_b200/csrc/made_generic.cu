@@ -358,13 +358,11 @@ struct GenericEngine {
     __device__ bool barrier() { return grid_barrier(r.ctl, epoch, r.spin_limit); }
     __device__ void init(const uint8_t *src) { init_phase<T>(m, r, src); }
     __device__ int compact(int) { return 0; }      // the CUDA-core path keeps the batch as it is
-    __device__ bool forward_logits(float *zout)
+    // one forward pass over the window; then either the logits go to zout (teacher forcing) or
+    // positions [w.plo, w.phi) are sampled and committed
+    __device__ bool step(const Win &w, bool flag, int parity, float *zout)
     {
-        const Win w = make_win(0, m.T, 0, m.T);
-        return forward_pass<T>(s, m, r, acts, zout, w, epoch, issued, skipped);
-    }
-    __device__ bool step(const Win &w, bool flag, int parity)
-    {
+        if (zout) return forward_pass<T>(s, m, r, acts, zout, w, epoch, issued, skipped);
         if (!forward_pass<T>(s, m, r, acts, m.logits, w, epoch, issued, skipped)) return false;
         sample_phase<T>(m, r, m.logits, w.plo, w.phi, flag, parity);
         return barrier();

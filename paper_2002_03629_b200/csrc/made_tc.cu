@@ -42,6 +42,7 @@ struct TcShared {
     uint32_t tmem_base;
     int off[JS_MAXL + 1];          // start of layer l's tile metadata inside `meta`
     float bias_s[4][256];          // per epilogue warp: bias of the current tile's columns
+    int sb_s[4][32];               // per epilogue warp: row -> sample index of the current tile (-1: none)
     int wcnt[NTH / 32];            // compaction: per-warp counts
     int cbase;                     // compaction: rows kept so far
 };
@@ -305,127 +306,155 @@ struct TcEngine {
         if (lane == 0) mbar_arrive(&sh.tempty[acc]);
     }
 
-    // hidden layer: act(acc + bias) -> bf16, 128 columns
+    // accumulator columns [half*64, half*64+64) of this warp's 32 rows -> staging, raw fp32,
+    // row-per-lane (thread = TMEM lane), 16-byte chunks swizzled by row
+    __device__ void stage_half(uint32_t tbase, int half)
+    {
+        uint8_t *stg = my_staging();
+        uint32_t ra[32], rb[32];
+        tmem_ld32_issue(tbase + (uint32_t)(half * 64), ra);       // two loads in flight per wait
+        tmem_ld32_issue(tbase + (uint32_t)(half * 64 + 32), rb);
+        tmem_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            *reinterpret_cast<uint4 *>(stg + lane * 256 + ((i ^ (lane & 15)) << 4)) =
+                make_uint4(ra[4 * i], ra[4 * i + 1], ra[4 * i + 2], ra[4 * i + 3]);
+            *reinterpret_cast<uint4 *>(stg + lane * 256 + (((i + 8) ^ (lane & 15)) << 4)) =
+                make_uint4(rb[4 * i], rb[4 * i + 1], rb[4 * i + 2], rb[4 * i + 3]);
+        }
+    }
+
+    // The row-wise passes below give half a warp to each row: lane -> row pair member (lane >> 4)
+    // and 16-byte chunk (lane & 15) = four consecutive columns.  Their loops are kept rolled: these
+    // kernels are instruction-cache bound when every path is unrolled.
+
+    // hidden layer: act(acc + bias) -> bf16, 128 columns in two halves of 64
     __device__ void epi_hidden_tile(int l, int mt, int n0, uint32_t tbase)
     {
         uint8_t *stg = my_staging();
         const float *bs = sh.bias_s[warp - 2];
-#pragma unroll 1
-        for (int c0 = 0; c0 < 128; c0 += 32) {
-            float v[32];
-            tmem_ld32(tbase + (uint32_t)c0, v);
-            uint32_t pk[16];
-#pragma unroll
-            for (int i = 0; i < 32; i += 2)
-                pk[i / 2] = pack_bf16x2(js_act_fn(m.act, v[i] + bs[c0 + i]), js_act_fn(m.act, v[i + 1] + bs[c0 + i + 1]));
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const int chunk = c0 / 8 + i;
-                *reinterpret_cast<uint4 *>(stg + lane * 256 + ((chunk ^ (lane & 15)) << 4)) =
-                    make_uint4(pk[4 * i], pk[4 * i + 1], pk[4 * i + 2], pk[4 * i + 3]);
-            }
-        }
-        release_acc();          // all TMEM reads of this tile are done (and the warp is in step)
-        if (warp == 2 && lane == 0) trace(6);
         const int N = m.n[l + 1];
         __nv_bfloat16 *out = (__nv_bfloat16 *)m.a[l + 1];
-        const int q = warp & 3, ch = lane & 15;
-        const int col = n0 + ch * 8;
-#pragma unroll 4
-        for (int it = 0; it < 16; ++it) {
-            const int rl = it * 2 + (lane >> 4);
-            const uint4 val = *reinterpret_cast<const uint4 *>(stg + rl * 256 + ((ch ^ (rl & 15)) << 4));
-            const int row = mt * BM + q * 32 + rl;
-            if (row < live && col < N) *reinterpret_cast<uint4 *>(out + (size_t)row * N + col) = val;
+        const int q = warp & 3, ch = lane & 15, rsel = lane >> 4;
+        const int act = m.act;
+#pragma unroll 1
+        for (int half = 0; half < 2; ++half) {
+            stage_half(tbase, half);
+            if (half == 1) { release_acc(); if (warp == 2 && lane == 0) trace(6); } else __syncwarp();
+            const int cb = half * 64 + ch * 4;
+            const float b0 = bs[cb], b1 = bs[cb + 1], b2 = bs[cb + 2], b3 = bs[cb + 3];
+            const int col = n0 + cb;
+#pragma unroll 2
+            for (int it = 0; it < 16; ++it) {
+                const int rl = it * 2 + rsel;
+                const float4 v = *reinterpret_cast<const float4 *>(stg + rl * 256 + ((ch ^ (rl & 15)) << 4));
+                const int row = mt * BM + q * 32 + rl;
+                const uint32_t p0 = pack_bf16x2(js_act_fn(act, v.x + b0), js_act_fn(act, v.y + b1));
+                const uint32_t p1 = pack_bf16x2(js_act_fn(act, v.z + b2), js_act_fn(act, v.w + b3));
+                if (row < live && col < N) *reinterpret_cast<uint2 *>(out + (size_t)row * N + col) = make_uint2(p0, p1);
+            }
+            __syncwarp();
         }
-        __syncwarp();
     }
 
-    // binary output layer: 128 positions per tile, handled as two halves of 64
+    // raise the per-sample change flag without hammering it: thousands of tiles report on the same
+    // few words, and stores to one address serialise in L2, so look first and store only if needed
+    __device__ void raise_flag(int parity, int sample)
+    {
+        int *f = &r.smp_changed[parity * r.batch + sample];
+        if (ld_volatile_i32(f) == 0) *f = 1;
+    }
+
+    // start this warp's rows of noise and symbols of a binary output tile towards L2 while the
+    // accumulator is still being computed (lane = row)
+    __device__ void bin_prefetch(int sample, int n0)
+    {
+        if (sample < 0 || n0 >= m.T) return;
+        const size_t at = (size_t)sample * m.T + n0;
+        const int ncols = min(128, m.T - n0);
+        for (int c = 0; c < ncols; c += 32) prefetch_l2(r.noise + at + c);
+        prefetch_l2(r.x + at);
+    }
+
+    // binary output layer: 128 positions per tile in two halves of 64: threshold the logit against
+    // the fixed noise, compare with the current symbol, commit symbol and encoding, note changes
     __device__ void epi_binary_tile(const Win &w, int mt, int n0, uint32_t tbase, bool flag, int parity,
                                     bool &wany, int &wfirst)
     {
         uint8_t *stg = my_staging();
         const float *bs = sh.bias_s[warp - 2];
-        const int T_ = m.T, q = warp & 3;
+        const int *sbs = sh.sb_s[warp - 2];
+        const int T_ = m.T, q = warp & 3, ch = lane & 15, rsel = lane >> 4;
         __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
         const float lut0 = m.lut[0], lut1 = m.lut[1];
-        const int *pm = perm_cur();
+        unsigned chmask = 0;           // rows of this warp with a change (bit = row)
+        int lfirst = INT_MAX;          // this lane's smallest changed position
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
-#pragma unroll 1
-            for (int cc = 0; cc < 2; ++cc) {
-                const int c0 = half * 64 + cc * 32;
-                float v[32];
-                tmem_ld32(tbase + (uint32_t)c0, v);
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int chunk = cc * 8 + i;
-                    *reinterpret_cast<float4 *>(stg + lane * 256 + ((chunk ^ (lane & 15)) << 4)) =
-                        make_float4(v[4 * i] + bs[c0 + 4 * i], v[4 * i + 1] + bs[c0 + 4 * i + 1],
-                                    v[4 * i + 2] + bs[c0 + 4 * i + 2], v[4 * i + 3] + bs[c0 + 4 * i + 3]);
-                }
-            }
+            stage_half(tbase, half);
             if (half == 1) release_acc(); else __syncwarp();
-            const int dbase = n0 + half * 64;
-            const int d = dbase + 2 * lane;                      // this lane's two positions d, d+1
-            const bool half_live = dbase < w.phi && dbase + 64 > w.plo && dbase < T_;
-            if (half_live) {
-                const bool in0 = d >= w.plo && d < w.phi && d < T_;
-                const bool in1 = d + 1 >= w.plo && d + 1 < w.phi && d + 1 < T_;
+            const int cb = half * 64 + ch * 4;
+            const int d = n0 + cb;                               // this lane's four positions d..d+3
+            unsigned inm = 0;                                    // which of them are inside the window
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (d + j >= w.plo && d + j < w.phi && d + j < T_) inm |= 1u << j;
+            const float b0 = bs[cb], b1 = bs[cb + 1], b2 = bs[cb + 2], b3 = bs[cb + 3];
 #pragma unroll 1
-                for (int g = 0; g < 32; g += 8) {
-                    const int row0 = mt * BM + q * 32 + g;
-                    if (row0 >= live) break;
-                    // issue the loads of eight rows together: the loop is latency-bound otherwise
-                    int sb[8];
+            for (int g = 0; g < 16; g += 4) {
+                // loads of eight rows in one go, then the decisions
+                float4 nz[4];
+                uint32_t xo[4];
+                int sb[4];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) sb[j] = row0 + j < live ? pm[row0 + j] : 0;
-                    float2 nz[8];
-                    unsigned short xo[8];
+                for (int j = 0; j < 4; ++j) {
+                    const int rl = (g + j) * 2 + rsel;
+                    sb[j] = sbs[rl];
+                    nz[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                    xo[j] = 0;
+                    if (sb[j] >= 0 && inm != 0u) {
+                        const size_t at = (size_t)sb[j] * T_ + d;
+                        nz[j] = __ldg(reinterpret_cast<const float4 *>(r.noise + at));
+                        xo[j] = *reinterpret_cast<const uint32_t *>(r.x + at);
+                    }
+                }
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        nz[j] = make_float2(0.0f, 0.0f);
-                        xo[j] = 0;
-                        if (row0 + j < live && (in0 || in1)) {
-                            const size_t at = (size_t)sb[j] * T_ + d;
-                            nz[j] = __ldg(reinterpret_cast<const float2 *>(r.noise + at));
-                            xo[j] = *reinterpret_cast<const unsigned short *>(r.x + at);
+                for (int j = 0; j < 4; ++j) {
+                    const int rl = (g + j) * 2 + rsel;
+                    const float4 v = *reinterpret_cast<const float4 *>(stg + rl * 256 + ((ch ^ (rl & 15)) << 4));
+                    bool changed = false;
+                    if (sb[j] >= 0 && inm != 0u) {
+                        const float z[4] = {v.x + b0, v.y + b1, v.z + b2, v.w + b3};
+                        const float e[4] = {nz[j].x, nz[j].y, nz[j].z, nz[j].w};
+                        uint32_t xn = 0;
+                        float enc[4];
+#pragma unroll
+                        for (int c = 0; c < 4; ++c) {
+                            const uint32_t o = (xo[j] >> (8 * c)) & 0xffu;
+                            const uint32_t nv = ((inm >> c) & 1u) ? (uint32_t)js_sample_binary(r.nk, z[c], e[c]) : o;
+                            if (nv != o && d + c < lfirst) lfirst = d + c;
+                            xn |= nv << (8 * c);
+                            enc[c] = nv ? lut1 : lut0;
+                        }
+                        changed = xn != xo[j];
+                        if (changed) {
+                            *reinterpret_cast<uint32_t *>(r.x + (size_t)sb[j] * T_ + d) = xn;
+                            const int row = mt * BM + q * 32 + rl;
+                            *reinterpret_cast<uint2 *>(a0 + (size_t)row * T_ + d) =
+                                make_uint2(pack_bf16x2(enc[0], enc[1]), pack_bf16x2(enc[2], enc[3]));
                         }
                     }
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        const int rl = g + j, row = row0 + j;
-                        if (row >= live) break;
-                        const float2 z = *reinterpret_cast<const float2 *>(
-                            stg + rl * 256 + ((((lane >> 1) ^ (rl & 15))) << 4) + (lane & 1) * 8);
-                        bool c0 = false, c1 = false;
-                        if (in0 || in1) {
-                            const size_t at = (size_t)sb[j] * T_ + d;
-                            const uint32_t o0 = xo[j] & 0xffu, o1 = xo[j] >> 8;
-                            const uint32_t n0v = in0 ? (uint32_t)js_sample_binary(r.nk, z.x, nz[j].x) : o0;
-                            const uint32_t n1v = in1 ? (uint32_t)js_sample_binary(r.nk, z.y, nz[j].y) : o1;
-                            c0 = n0v != o0;
-                            c1 = n1v != o1;
-                            if (c0 || c1) {
-                                *reinterpret_cast<unsigned short *>(r.x + at) = (unsigned short)(n0v | (n1v << 8));
-                                *reinterpret_cast<uint32_t *>(a0 + (size_t)row * T_ + d) =
-                                    pack_bf16x2(n0v ? lut1 : lut0, n1v ? lut1 : lut0);
-                            }
-                        }
-                        const unsigned bal = __ballot_sync(0xffffffffu, c0 || c1);
-                        if (bal != 0u && flag) {
-                            const int fl = __ffs(bal) - 1;
-                            const int fc0 = __shfl_sync(0xffffffffu, (int)c0, fl);
-                            const int fd = dbase + 2 * fl + (fc0 ? 0 : 1);
-                            if (lane == 0) r.smp_changed[parity * r.batch + sb[j]] = 1;
-                            wany = true;
-                            wfirst = min(wfirst, fd);
-                        }
-                    }
+                    const unsigned bal = __ballot_sync(0xffffffffu, changed);
+                    if (bal & 0x0000ffffu) chmask |= 1u << ((g + j) * 2);
+                    if (bal & 0xffff0000u) chmask |= 1u << ((g + j) * 2 + 1);
                 }
             }
             __syncwarp();
+        }
+        if (flag && chmask != 0u) {
+            if (((chmask >> lane) & 1u) && sbs[lane] >= 0) raise_flag(parity, sbs[lane]);      // lane = row
+            wany = true;
+            wfirst = min(wfirst, __reduce_min_sync(0xffffffffu, lfirst));
         }
     }
 
@@ -439,6 +468,14 @@ struct TcEngine {
         for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
             const int nt = nt_lo + id / MT, mt = id % MT;
             if (kind == EPI_HIDDEN || kind == EPI_BINARY) load_bias_tile(l, nt * ly.bn, ly.bn);
+            if (kind == EPI_BINARY) {
+                const int rw = mt * BM + q * 32 + lane;
+                const int smp = rw < live ? perm_cur()[rw] : -1;
+                __syncwarp();
+                sh.sb_s[warp - 2][lane] = smp;
+                __syncwarp();
+                bin_prefetch(smp, nt * ly.bn);              // in flight while the tile is still being computed
+            }
             if (!mbar_wait(&sh.tfull[acc], aphase, r.ctl)) { dead = true; break; }
             tc_fence_after();
             if (warp == 2 && lane == 0) trace(3);
@@ -474,7 +511,7 @@ struct TcEngine {
                     }
                 }
                 if (flag && ch) {
-                    r.smp_changed[parity * r.batch + sample] = 1;
+                    raise_flag(parity, sample);
                     any_changed = true;
                     first = min(first, fc);
                 }
@@ -521,24 +558,18 @@ struct TcEngine {
         return true;
     }
 
-    __device__ bool forward_logits(float *zout)
+    // one forward pass over the window: a single loop and a single call site, so that the whole
+    // pipeline is instantiated once in the kernel
+    __device__ bool step(const Win &w, bool flag, int parity, float *zout)
     {
-        const Win w = make_win(0, m.T, 0, m.T);
-        for (int l = 0; l < m.L; ++l) {
-            gemm_phase(l, EPI_HIDDEN, w, false, 0, nullptr);
-            if (!barrier()) return false;
-        }
-        gemm_phase(m.L, EPI_LOGITS, w, false, 0, zout);
-        return barrier();
-    }
-
-    __device__ bool step(const Win &w, bool flag, int parity)
-    {
-        for (int l = 0; l < m.L; ++l)
-            if (gemm_phase(l, EPI_HIDDEN, w, false, 0, nullptr))
+        const int out_kind = zout ? EPI_LOGITS : (m.C == 1 ? EPI_BINARY : EPI_CAT);
+        for (int l = 0; l <= m.L; ++l) {
+            const bool last = (l == m.L);
+            const bool did = gemm_phase(l, last ? out_kind : EPI_HIDDEN, w, last && flag, parity, zout);
+            if (did || last)
                 if (!barrier()) return false;
-        gemm_phase(m.L, m.C == 1 ? EPI_BINARY : EPI_CAT, w, flag, parity, nullptr);
-        return barrier();
+        }
+        return true;
     }
 };
 
