@@ -14,12 +14,23 @@ struct TcLayer {
     const int *dmax;
     int bn;
     int nt;
+    // split-K: the K blocks of tile nt are cut into chunks of `ch` blocks, each chunk a work unit
+    // of its own; the last chunk owns the tile and adds the others' fp32 partial sums in order
+    int ch;
+    int slots_per_mt;            // partial-sum slots per row tile = sum over nt of (chunks - 1)
+    const int *slot_base;        // [nt] first slot of tile nt inside a row tile
+    const int *sched_off;        // [grid + 1] work units of CTA c: sched[sched_off[c] .. sched_off[c+1])
+    const int *sched;            // units packed as (row tile << 24) | (n tile << 8) | chunk
 };
 struct TcDev {
     const CUtensorMap *tmA;      // [L+1] activations a[l], box 64 x 128
     const CUtensorMap *tmW;      // [L+1] masked weights W[l], box 64 x bn
     TcLayer lay[JS_MAXL + 1];
     int stage_bytes, n_stages, smem_bytes;
+    int grid;                    // CTAs the schedules were built for (the launch uses exactly this)
+    float *partials;             // [slot][columns/4][128 rows] float4: fp32 partial sums of non-owning chunks
+    unsigned *pflags;            // [slot][4 row quadrants]: phase stamp once the partial is stored
+    int n_pflags;
 };
 
 // Device view of a masked-convolution stack (tensor-core kernel only).

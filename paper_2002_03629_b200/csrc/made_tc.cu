@@ -18,6 +18,10 @@
 // drains, TMEM is freed and the kernel returns JS_ERR_TIMEOUT.
 #include <cuda.h>
 
+#include <algorithm>
+#include <cstdio>
+#include <cstdlib>
+
 #include "js_common.cuh"
 #include "js_model.h"
 #include "made_driver.cuh"
@@ -82,6 +86,11 @@ struct TcEngine {
     __device__ const int *perm_cur() const { return r.perm + (size_t)pcur * r.perm_stride; }
 
     int phase_no = 0;              // counts gemm phases, for the optional timeline
+    unsigned stamp = 0;            // phase counter: marks this phase's partial-sum flags
+    // partial sums the tile being finished has to add (owner chunk): set per tile by the epilogue
+    int cur_parts = 0;
+    const float *cur_pbase = nullptr;
+    size_t cur_tile_floats = 0;
     __device__ void trace(int slot) const
     {
         if (r.trace == nullptr || phase_no >= JS_TRACE_PHASES) return;
@@ -109,6 +118,9 @@ struct TcEngine {
             if (r.x) r.x[i] = v;
             a0[i] = __float2bfloat16_rn(m.lut[v]);
         }
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)t.n_pflags;
+             i += (size_t)gridDim.x * blockDim.x)
+            t.pflags[i] = 0u;
         if (blockIdx.x == 0) {
             for (int i = threadIdx.x; i < 2 * r.batch; i += blockDim.x) {
                 r.smp_changed[i] = 0;
@@ -203,45 +215,81 @@ struct TcEngine {
         nt_hi = a;
     }
 
-    __device__ void producer(int l, int nt_lo, int ntiles, int MT)
+    // ---- work units.  The K blocks of a tile are cut into chunks of ly.ch blocks (a property of
+    // the layer and the tile alone, never of the window, so that every value is always summed
+    // in the same order).  Each chunk is a unit; the host gave every CTA its list of units,
+    // balanced by K length, non-owning chunks first.  The chunk with the highest K blocks owns
+    // the tile: it adds the other chunks' fp32 partial sums in chunk order and runs the epilogue.
+    // Because every CTA works through partial chunks before owners, an owner's wait always ends.
+    struct Unit {
+        int mt, nt, kb0, kb1;
+        int nparts;        // owner: partial sums to add (>= 0); non-owner: -1
+        int slot;          // non-owner: its slot; owner: slot of the tile's first partial
+    };
+    __device__ bool next_unit(int l, int &e, int e_end, int nt_lo, int nt_hi, int MT, Unit &u) const
+    {
+        const TcLayer &ly = t.lay[l];
+        while (e < e_end) {
+            const int v = ly.sched[e++];
+            u.mt = v >> 24;
+            u.nt = (v >> 8) & 0xffff;
+            const int chunk = v & 0xff;
+            if (u.mt >= MT || u.nt < nt_lo || u.nt >= nt_hi) continue;
+            const int kbe = kb_end_of(l, u.nt);
+            const int nc = (kbe + ly.ch - 1) / ly.ch;
+            u.kb0 = chunk * ly.ch;
+            u.kb1 = min(kbe, u.kb0 + ly.ch);
+            const bool owner = (chunk == nc - 1);
+            u.nparts = owner ? nc - 1 : -1;
+            u.slot = u.mt * ly.slots_per_mt + ly.slot_base[u.nt] + (owner ? 0 : chunk);
+            return true;
+        }
+        return false;
+    }
+
+    __device__ void producer(int l, int nt_lo, int nt_hi, int MT)
     {
         const TcLayer &ly = t.lay[l];
         const CUtensorMap *ma = t.tmA + l, *mw = t.tmW + l;
         const uint32_t bytes = A_BYTES + ly.bn * BK * 2;
         trace(0);
-        for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
-            const int nt = nt_lo + id / MT, mt = id % MT;
-            const int kb_end = kb_end_of(l, nt);
-            for (int kb = 0; kb < kb_end; ++kb) {
+        int e = ly.sched_off[blockIdx.x];
+        const int e_end = ly.sched_off[blockIdx.x + 1];
+        Unit u;
+        while (!dead && next_unit(l, e, e_end, nt_lo, nt_hi, MT, u)) {
+            issued++;
+            for (int kb = u.kb0; kb < u.kb1; ++kb) {
                 if (!mbar_wait(&sh.empty[stage], sphase ^ 1u, r.ctl)) { dead = true; break; }
                 mbar_expect_tx(&sh.full[stage], bytes);
-                tma_load_2d(smem_u32(stage_a(stage)), ma, &sh.full[stage], kb * BK, mt * BM);
-                tma_load_2d(smem_u32(stage_b(stage)), mw, &sh.full[stage], kb * BK, nt * ly.bn);
+                tma_load_2d(smem_u32(stage_a(stage)), ma, &sh.full[stage], kb * BK, u.mt * BM);
+                tma_load_2d(smem_u32(stage_b(stage)), mw, &sh.full[stage], kb * BK, u.nt * ly.bn);
                 advance_stage();
             }
         }
     }
 
-    __device__ void mma_issuer(int l, int nt_lo, int ntiles, int MT)
+    __device__ void mma_issuer(int l, int nt_lo, int nt_hi, int MT)
     {
         const TcLayer &ly = t.lay[l];
         const uint32_t idesc = instr_desc_bf16(ly.bn);
-        for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
-            const int nt = nt_lo + id / MT;
-            const int kb_end = kb_end_of(l, nt);
+        int e = ly.sched_off[blockIdx.x];
+        const int e_end = ly.sched_off[blockIdx.x + 1];
+        Unit u;
+        bool first = true;
+        while (!dead && next_unit(l, e, e_end, nt_lo, nt_hi, MT, u)) {
             if (!mbar_wait(&sh.tempty[acc], aphase ^ 1u, r.ctl)) { dead = true; break; }
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_COLS);
-            for (int kb = 0; kb < kb_end; ++kb) {
+            for (int kb = u.kb0; kb < u.kb1; ++kb) {
                 if (!mbar_wait(&sh.full[stage], sphase, r.ctl)) { dead = true; break; }
                 tc_fence_after();
-                if (kb == 0 && id == (int)blockIdx.x) trace(1);
+                if (first) { trace(1); first = false; }
                 const uint64_t adesc = smem_desc_sw128(smem_u32(stage_a(stage)));
                 const uint64_t bdesc = smem_desc_sw128(smem_u32(stage_b(stage)));
 #pragma unroll
                 for (int k = 0; k < BK / 16; ++k)       // 16 bf16 = 32 bytes per instruction along K
                     umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
-                              (kb > 0 || k > 0) ? 1u : 0u);
+                              (kb > u.kb0 || k > 0) ? 1u : 0u);
                 umma_commit(&sh.empty[stage]);          // frees the stage once these MMAs have read it
                 advance_stage();
             }
@@ -250,6 +298,101 @@ struct TcEngine {
             advance_acc();
         }
         trace(2);
+    }
+
+    // ---- partial sums.  Layout of a slot: [column / 4][128 rows] float4, written and read with
+    // thread = row, so stores and loads are coalesced without any transposition.
+    __device__ size_t tile_floats(int l) const { return (size_t)BM * t.lay[l].bn; }
+
+    // non-owning chunk: accumulator -> its slot, then raise the slot's flag for this row quadrant
+    __device__ void store_partial(int l, int slot, uint32_t tbase)
+    {
+        const int q = warp & 3, row = q * 32 + lane;
+        float4 *base = reinterpret_cast<float4 *>(t.partials + (size_t)slot * tile_floats(l)) + row;
+#pragma unroll 1
+        for (int c0 = 0; c0 < t.lay[l].bn; c0 += 32) {
+            uint32_t ra[32];
+            tmem_ld32_issue(tbase + (uint32_t)c0, ra);
+            tmem_wait_ld();
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                base[(size_t)(c0 / 4 + i) * BM] = make_float4(__uint_as_float(ra[4 * i]), __uint_as_float(ra[4 * i + 1]),
+                                                              __uint_as_float(ra[4 * i + 2]), __uint_as_float(ra[4 * i + 3]));
+        }
+        release_acc();
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) {
+            unsigned *f = t.pflags + (size_t)slot * 4 + q;
+            asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(f), "r"(stamp) : "memory");
+        }
+    }
+
+    // owner: bounded wait until this warp's row quadrant of every partial of the tile is stored
+    __device__ bool wait_partials(int slot, int nparts)
+    {
+        int ok = 1;
+        if (lane == 0) {
+            const int q = warp & 3;
+            for (int p = 0; p < nparts && ok; ++p) {
+                const unsigned *f = t.pflags + (size_t)(slot + p) * 4 + q;
+                uint64_t t0 = 0;
+                for (unsigned i = 0; ld_acquire_u32(f) != stamp; ++i) {
+                    if ((i & 15u) == 15u) {
+                        if (t0 == 0) t0 = global_ns();
+                        if (ld_volatile_i32(&r.ctl->abort) != 0 || global_ns() - t0 > MBAR_WAIT_NS) {
+                            atomicExch(&r.ctl->abort, 1);
+                            ok = 0;
+                            break;
+                        }
+                    }
+                }
+            }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        __threadfence();
+        return ok != 0;
+    }
+
+    // the same for 64 columns held in two register groups, with all sixteen loads of a partial in
+    // flight together (one memory latency per partial instead of two)
+    __device__ void add_partials64(uint32_t (&ra)[32], uint32_t (&rb)[32], int c0) const
+    {
+        const int row = (warp & 3) * 32 + lane;
+        for (int p = 0; p < cur_parts; ++p) {
+            const float4 *base = reinterpret_cast<const float4 *>(cur_pbase + (size_t)p * cur_tile_floats) + row;
+            float4 v[16];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = __ldcg(base + (size_t)(c0 / 4 + i) * BM);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                ra[4 * i] = __float_as_uint(__uint_as_float(ra[4 * i]) + v[i].x);
+                ra[4 * i + 1] = __float_as_uint(__uint_as_float(ra[4 * i + 1]) + v[i].y);
+                ra[4 * i + 2] = __float_as_uint(__uint_as_float(ra[4 * i + 2]) + v[i].z);
+                ra[4 * i + 3] = __float_as_uint(__uint_as_float(ra[4 * i + 3]) + v[i].w);
+                rb[4 * i] = __float_as_uint(__uint_as_float(rb[4 * i]) + v[i + 8].x);
+                rb[4 * i + 1] = __float_as_uint(__uint_as_float(rb[4 * i + 1]) + v[i + 8].y);
+                rb[4 * i + 2] = __float_as_uint(__uint_as_float(rb[4 * i + 2]) + v[i + 8].z);
+                rb[4 * i + 3] = __float_as_uint(__uint_as_float(rb[4 * i + 3]) + v[i + 8].w);
+            }
+        }
+    }
+
+    // add the tile's partial sums, in chunk order, to 32 accumulator columns starting at c0
+    __device__ void add_partials(uint32_t (&ra)[32], int c0) const
+    {
+        const int row = (warp & 3) * 32 + lane;
+        for (int p = 0; p < cur_parts; ++p) {
+            const float4 *base = reinterpret_cast<const float4 *>(cur_pbase + (size_t)p * cur_tile_floats) + row;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float4 v = __ldcg(base + (size_t)(c0 / 4 + i) * BM);
+                ra[4 * i] = __float_as_uint(__uint_as_float(ra[4 * i]) + v.x);
+                ra[4 * i + 1] = __float_as_uint(__uint_as_float(ra[4 * i + 1]) + v.y);
+                ra[4 * i + 2] = __float_as_uint(__uint_as_float(ra[4 * i + 2]) + v.z);
+                ra[4 * i + 3] = __float_as_uint(__uint_as_float(ra[4 * i + 3]) + v.w);
+            }
+        }
     }
 
     // ---- chunk-wise epilogues: thread = one sample row of the tile, 32 columns at a time
@@ -315,6 +458,7 @@ struct TcEngine {
         tmem_ld32_issue(tbase + (uint32_t)(half * 64), ra);       // two loads in flight per wait
         tmem_ld32_issue(tbase + (uint32_t)(half * 64 + 32), rb);
         tmem_wait_ld();
+        if (cur_parts > 0) add_partials64(ra, rb, half * 64);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             *reinterpret_cast<uint4 *>(stg + lane * 256 + ((i ^ (lane & 15)) << 4)) =
@@ -344,7 +488,7 @@ struct TcEngine {
             const int cb = half * 64 + ch * 4;
             const float b0 = bs[cb], b1 = bs[cb + 1], b2 = bs[cb + 2], b3 = bs[cb + 3];
             const int col = n0 + cb;
-#pragma unroll 2
+#pragma unroll 4
             for (int it = 0; it < 16; ++it) {
                 const int rl = it * 2 + rsel;
                 const float4 v = *reinterpret_cast<const float4 *>(stg + rl * 256 + ((ch ^ (rl & 15)) << 4));
@@ -378,79 +522,101 @@ struct TcEngine {
 
     // binary output layer: 128 positions per tile in two halves of 64: threshold the logit against
     // the fixed noise, compare with the current symbol, commit symbol and encoding, note changes
+    // noise and current symbols of eight row pairs (rows (g+j)*2 + rsel) at this lane's four positions
+    struct BinRows {
+        float4 nz[8];
+        uint32_t xo[8];
+        int sb[8];
+    };
+    __device__ void bin_load_rows(BinRows &in, const int *sbs, int g, int d, bool any_in) const
+    {
+        const int rsel = lane >> 4;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int rl = (g + j) * 2 + rsel;
+            in.sb[j] = sbs[rl];
+            in.nz[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+            in.xo[j] = 0;
+            if (in.sb[j] >= 0 && any_in) {
+                const size_t at = (size_t)in.sb[j] * m.T + d;
+                in.nz[j] = ld_nc_f4_now(r.noise + at);      // issued here, not at first use
+                in.xo[j] = ld_u32_now(r.x + at);
+            }
+        }
+    }
+    __device__ void bin_decide_rows(const BinRows &in, int g, int mt, int d, unsigned inm, const float (&bias4)[4],
+                                    unsigned &chmask, int &lfirst)
+    {
+        uint8_t *stg = my_staging();
+        const int q = warp & 3, ch = lane & 15, rsel = lane >> 4, T_ = m.T;
+        __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
+        const float lut0 = m.lut[0], lut1 = m.lut[1];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int rl = (g + j) * 2 + rsel;
+            const float4 v = *reinterpret_cast<const float4 *>(stg + rl * 256 + ((ch ^ (rl & 15)) << 4));
+            bool changed = false;
+            if (in.sb[j] >= 0 && inm != 0u) {
+                const float z[4] = {v.x + bias4[0], v.y + bias4[1], v.z + bias4[2], v.w + bias4[3]};
+                const float e[4] = {in.nz[j].x, in.nz[j].y, in.nz[j].z, in.nz[j].w};
+                uint32_t xn = 0;
+                float enc[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t o = (in.xo[j] >> (8 * c)) & 0xffu;
+                    const uint32_t nv = ((inm >> c) & 1u) ? (uint32_t)js_sample_binary(r.nk, z[c], e[c]) : o;
+                    if (nv != o && d + c < lfirst) lfirst = d + c;
+                    xn |= nv << (8 * c);
+                    enc[c] = nv ? lut1 : lut0;
+                }
+                changed = xn != in.xo[j];
+                if (changed) {
+                    *reinterpret_cast<uint32_t *>(r.x + (size_t)in.sb[j] * T_ + d) = xn;
+                    const int row = mt * BM + q * 32 + rl;
+                    *reinterpret_cast<uint2 *>(a0 + (size_t)row * T_ + d) =
+                        make_uint2(pack_bf16x2(enc[0], enc[1]), pack_bf16x2(enc[2], enc[3]));
+                }
+            }
+            // bit = row of the warp; no warp vote here, so that the eight iterations can overlap
+            if (changed) chmask |= 1u << rl;
+        }
+    }
+
+    // binary output layer: 128 positions per tile in two halves of 64: threshold the logit against
+    // the fixed noise, compare with the current symbol, commit symbol and encoding, note changes.
+    // The loads of a half's first sixteen rows are issued before the accumulator is staged, those of
+    // the other sixteen before the first ones are used, so that little memory latency stays exposed.
     __device__ void epi_binary_tile(const Win &w, int mt, int n0, uint32_t tbase, bool flag, int parity,
                                     bool &wany, int &wfirst)
     {
-        uint8_t *stg = my_staging();
         const float *bs = sh.bias_s[warp - 2];
         const int *sbs = sh.sb_s[warp - 2];
-        const int T_ = m.T, q = warp & 3, ch = lane & 15, rsel = lane >> 4;
-        __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
-        const float lut0 = m.lut[0], lut1 = m.lut[1];
-        unsigned chmask = 0;           // rows of this warp with a change (bit = row)
+        const int T_ = m.T, ch = lane & 15;
+        unsigned chmask = 0;           // rows in which this lane changed something (bit = row of the warp)
         int lfirst = INT_MAX;          // this lane's smallest changed position
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
-            stage_half(tbase, half);
-            if (half == 1) release_acc(); else __syncwarp();
             const int cb = half * 64 + ch * 4;
             const int d = n0 + cb;                               // this lane's four positions d..d+3
             unsigned inm = 0;                                    // which of them are inside the window
 #pragma unroll
             for (int j = 0; j < 4; ++j)
                 if (d + j >= w.plo && d + j < w.phi && d + j < T_) inm |= 1u << j;
-            const float b0 = bs[cb], b1 = bs[cb + 1], b2 = bs[cb + 2], b3 = bs[cb + 3];
-#pragma unroll 1
-            for (int g = 0; g < 16; g += 4) {
-                // loads of eight rows in one go, then the decisions
-                float4 nz[4];
-                uint32_t xo[4];
-                int sb[4];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int rl = (g + j) * 2 + rsel;
-                    sb[j] = sbs[rl];
-                    nz[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                    xo[j] = 0;
-                    if (sb[j] >= 0 && inm != 0u) {
-                        const size_t at = (size_t)sb[j] * T_ + d;
-                        nz[j] = __ldg(reinterpret_cast<const float4 *>(r.noise + at));
-                        xo[j] = *reinterpret_cast<const uint32_t *>(r.x + at);
-                    }
-                }
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int rl = (g + j) * 2 + rsel;
-                    const float4 v = *reinterpret_cast<const float4 *>(stg + rl * 256 + ((ch ^ (rl & 15)) << 4));
-                    bool changed = false;
-                    if (sb[j] >= 0 && inm != 0u) {
-                        const float z[4] = {v.x + b0, v.y + b1, v.z + b2, v.w + b3};
-                        const float e[4] = {nz[j].x, nz[j].y, nz[j].z, nz[j].w};
-                        uint32_t xn = 0;
-                        float enc[4];
-#pragma unroll
-                        for (int c = 0; c < 4; ++c) {
-                            const uint32_t o = (xo[j] >> (8 * c)) & 0xffu;
-                            const uint32_t nv = ((inm >> c) & 1u) ? (uint32_t)js_sample_binary(r.nk, z[c], e[c]) : o;
-                            if (nv != o && d + c < lfirst) lfirst = d + c;
-                            xn |= nv << (8 * c);
-                            enc[c] = nv ? lut1 : lut0;
-                        }
-                        changed = xn != xo[j];
-                        if (changed) {
-                            *reinterpret_cast<uint32_t *>(r.x + (size_t)sb[j] * T_ + d) = xn;
-                            const int row = mt * BM + q * 32 + rl;
-                            *reinterpret_cast<uint2 *>(a0 + (size_t)row * T_ + d) =
-                                make_uint2(pack_bf16x2(enc[0], enc[1]), pack_bf16x2(enc[2], enc[3]));
-                        }
-                    }
-                    const unsigned bal = __ballot_sync(0xffffffffu, changed);
-                    if (bal & 0x0000ffffu) chmask |= 1u << ((g + j) * 2);
-                    if (bal & 0xffff0000u) chmask |= 1u << ((g + j) * 2 + 1);
-                }
-            }
+            const float bias4[4] = {bs[cb], bs[cb + 1], bs[cb + 2], bs[cb + 3]};
+            BinRows ra, rb;
+            const bool tr = (warp == 2 && lane == 0);
+            if (tr) trace(6 + 3 * half);
+            bin_load_rows(ra, sbs, 0, d, inm != 0u);
+            stage_half(tbase, half);
+            if (half == 1) release_acc(); else __syncwarp();
+            if (tr) trace(7 + 3 * half);
+            bin_load_rows(rb, sbs, 8, d, inm != 0u);
+            bin_decide_rows(ra, 0, mt, d, inm, bias4, chmask, lfirst);
+            if (tr) trace(8 + 3 * half);
+            bin_decide_rows(rb, 8, mt, d, inm, bias4, chmask, lfirst);
             __syncwarp();
         }
+        chmask = __reduce_or_sync(0xffffffffu, chmask);           // rows changed by any lane
         if (flag && chmask != 0u) {
             if (((chmask >> lane) & 1u) && sbs[lane] >= 0) raise_flag(parity, sbs[lane]);      // lane = row
             wany = true;
@@ -459,16 +625,20 @@ struct TcEngine {
     }
 
     __device__ void epilogue(int l, int kind, const Win &w, bool flag, int parity, float *zout, int nt_lo,
-                             int ntiles, int MT)
+                             int nt_hi, int MT)
     {
         const TcLayer &ly = t.lay[l];
         const int q = warp & 3;
         bool any_changed = false;
         int first = INT_MAX;
-        for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
-            const int nt = nt_lo + id / MT, mt = id % MT;
-            if (kind == EPI_HIDDEN || kind == EPI_BINARY) load_bias_tile(l, nt * ly.bn, ly.bn);
-            if (kind == EPI_BINARY) {
+        int e = ly.sched_off[blockIdx.x];
+        const int e_end = ly.sched_off[blockIdx.x + 1];
+        Unit u;
+        while (!dead && next_unit(l, e, e_end, nt_lo, nt_hi, MT, u)) {
+            const int nt = u.nt, mt = u.mt;
+            const bool owner = u.nparts >= 0;
+            if (owner && (kind == EPI_HIDDEN || kind == EPI_BINARY)) load_bias_tile(l, nt * ly.bn, ly.bn);
+            if (owner && kind == EPI_BINARY) {
                 const int rw = mt * BM + q * 32 + lane;
                 const int smp = rw < live ? perm_cur()[rw] : -1;
                 __syncwarp();
@@ -482,6 +652,15 @@ struct TcEngine {
             const int row = mt * BM + q * 32 + lane;
             const int n0 = nt * ly.bn;
             const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS);
+            if (!owner) {
+                store_partial(l, u.slot, tbase);
+                advance_acc();
+                continue;
+            }
+            cur_parts = u.nparts;
+            cur_pbase = t.partials + (size_t)u.slot * tile_floats(l);
+            cur_tile_floats = tile_floats(l);
+            if (cur_parts > 0 && !wait_partials(u.slot, cur_parts)) { dead = true; break; }
             if (kind == EPI_HIDDEN) {
                 epi_hidden_tile(l, mt, n0, tbase);
             } else if (kind == EPI_BINARY) {
@@ -497,7 +676,14 @@ struct TcEngine {
                 const int sample = (kind == EPI_CAT && row < live) ? perm_cur()[row] : -1;
                 for (int c0 = 0; c0 < ly.bn; c0 += 32) {
                     float v[32];
-                    tmem_ld32(tbase + (uint32_t)c0, v);
+                    {
+                        uint32_t ra[32];
+                        tmem_ld32_issue(tbase + (uint32_t)c0, ra);
+                        tmem_wait_ld();
+                        if (cur_parts > 0) add_partials(ra, c0);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(ra[i]);
+                    }
                     if (kind == EPI_LOGITS) epi_logits(zout, row, n0, c0, v);
                     else epi_cat_chunk(sample, nt, c0, v, best, bi);
                 }
@@ -539,21 +725,16 @@ struct TcEngine {
         live_range(l, w, nt_lo, nt_hi);
         const int MT = (live + BM - 1) / BM;
         const int nlive = max(0, nt_hi - nt_lo);
-        const int ntiles = nlive * MT;
-        if (threadIdx.x == 0) {
-            int mine = 0;
-            for (int id = blockIdx.x; id < ntiles; id += gridDim.x) mine++;
-            issued += mine;
-            if (blockIdx.x == 0) skipped += (unsigned long long)(t.lay[l].nt - nlive) * MT;
-        }
-        if (ntiles == 0) return false;
+        if (threadIdx.x == 0 && blockIdx.x == 0) skipped += (unsigned long long)(t.lay[l].nt - nlive) * MT;
+        stamp += 1;
+        if (nlive == 0) return false;
         phase_no++;
         if (warp == 0) {
-            if (lane == 0) producer(l, nt_lo, ntiles, MT);
+            if (lane == 0) producer(l, nt_lo, nt_hi, MT);
         } else if (warp == 1) {
-            if (lane == 0) mma_issuer(l, nt_lo, ntiles, MT);
+            if (lane == 0) mma_issuer(l, nt_lo, nt_hi, MT);
         } else {
-            epilogue(l, kind, w, flag, parity, zout, nt_lo, ntiles, MT);
+            epilogue(l, kind, w, flag, parity, zout, nt_lo, nt_hi, MT);
         }
         return true;
     }
@@ -680,6 +861,7 @@ int js_tc_prepare(js_model *mo)
     t.n_stages = RING_BYTES / t.stage_bytes;
     if (t.n_stages > MAX_STAGES) t.n_stages = MAX_STAGES;
     std::vector<CUtensorMap> mapsA(L + 1), mapsW(L + 1);
+    std::vector<std::vector<int>> kb_all(L + 1);
     for (int l = 0; l <= L; ++l) {
         const int bn = (l == L && wide) ? 256 : 128;
         const int N = v.n[l + 1], K = v.n[l], nt = (N + bn - 1) / bn;
@@ -705,8 +887,153 @@ int js_tc_prepare(js_model *mo)
         }
         t.lay[l].bn = bn;
         t.lay[l].nt = nt;
+        kb_all[l] = kb;
         if (!encode_map(&mapsA[l], v.a[l], mo->rows, K, BM)) return 0;
         if (!encode_map(&mapsW[l], v.W[l], N, K, bn)) return 0;
+    }
+    // ---- split-K work units and their static assignment to CTAs (longest processing time first)
+    int sms = 0;
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (sms < 1) return 0;
+    }
+    const int MTmax = mo->rows / BM;
+    std::vector<int> chs(L + 1);
+    int G = 1;
+    for (int l = 0; l <= L; ++l) {
+        const std::vector<int> &kb = kb_all[l];
+        long long total_kb = 0;
+        for (int x : kb) total_kb += (long long)x * MTmax;
+        int ch = 1 << 20;                                              // enough tiles: no split
+        if ((long long)kb.size() * MTmax < 2LL * sms) {
+            // a CTA's fair share of the layer, but never less than half of the longest tile: every
+            // extra chunk costs its owner a 64 KB read of partial sums
+            int kb_max = 1;
+            for (int x : kb) kb_max = std::max(kb_max, x);
+            ch = (int)std::max<long long>(std::max<long long>(4, (kb_max + 1) / 2), (total_kb + sms - 1) / sms);
+        }
+        chs[l] = ch;
+        long long units = 0;
+        for (int x : kb) units += (long long)((x + ch - 1) / ch) * MTmax;
+        G = (int)std::max<long long>(G, std::min<long long>(sms, units));
+    }
+    t.grid = G;
+    size_t part_floats = 0;
+    int max_slots = 0;
+    for (int l = 0; l <= L; ++l) {
+        const std::vector<int> &kb = kb_all[l];
+        const int ch = chs[l], nt = (int)kb.size(), bn = t.lay[l].bn;
+        std::vector<int> slot_base(nt);
+        int slots = 0;
+        for (int i = 0; i < nt; ++i) { slot_base[i] = slots; slots += (kb[i] + ch - 1) / ch - 1; }
+        // units: non-owning chunks first (all of size ch), then owners by decreasing size
+        struct U { int mt, nt, chunk, size; };
+        std::vector<U> part, own;
+        for (int mt = 0; mt < MTmax; ++mt)
+            for (int i = 0; i < nt; ++i) {
+                const int nc = (kb[i] + ch - 1) / ch;
+                for (int c = 0; c + 1 < nc; ++c) part.push_back({mt, i, c, ch});
+                own.push_back({mt, i, nc - 1, kb[i] - ch * (nc - 1)});
+            }
+        // List scheduling on a small model of a CTA, in units of one K block's load time: the K
+        // loops of a CTA's units run back to back; a unit's epilogue starts when its K loop is
+        // done, the previous epilogue is done and (for an owner) the tile's partial sums have been
+        // stored.  Units are taken longest first and put where the CTA finishes earliest.  Inside
+        // a CTA: partial chunks first (owners elsewhere wait for them), then owners that wait for
+        // nobody, then owners that add partial sums.
+        const int EPI_PART = 7, EPI_OWN = (l == L ? 24 : 10), EPI_ADD = 7;
+        auto nparts_of = [&](const U &u) { return (kb[u.nt] + ch - 1) / ch - 1; };
+        struct Item { int code, size, epi, ready; };
+        std::vector<std::vector<Item>> lp(G), lo0(G), lo1(G);
+        auto finish = [&](int c, const Item *extra, int where) {
+            long long M = 2, E = 0;
+            auto run = [&](const Item &it) {
+                M += it.size;
+                const long long start = std::max<long long>(std::max(M, E), it.ready);
+                E = start + it.epi;
+            };
+            for (const Item &it : lp[c]) run(it);
+            if (extra && where == 0) run(*extra);
+            for (const Item &it : lo0[c]) run(it);
+            if (extra && where == 1) run(*extra);
+            for (const Item &it : lo1[c]) run(it);
+            if (extra && where == 2) run(*extra);
+            return E;
+        };
+        auto place = [&](const Item &it, int where) {
+            int best = 0;
+            long long bt = -1;
+            for (int c = 0; c < G; ++c) {
+                const long long f = finish(c, &it, where);
+                if (bt < 0 || f < bt) { bt = f; best = c; }
+            }
+            (where == 0 ? lp : where == 1 ? lo0 : lo1)[best].push_back(it);
+            return best;
+        };
+        std::vector<long long> ready((size_t)MTmax * nt, 0);          // when a tile's partial sums are all stored
+        for (const U &u : part) {
+            const Item it = {(u.mt << 24) | (u.nt << 8) | u.chunk, u.size, EPI_PART, 0};
+            const int c = place(it, 0);
+            long long M = 2, E = 0;                                    // completion of this chunk in its CTA
+            for (const Item &x : lp[c]) { M += x.size; E = std::max(M, E) + x.epi; }
+            ready[(size_t)u.mt * nt + u.nt] = std::max(ready[(size_t)u.mt * nt + u.nt], E);
+        }
+        std::stable_sort(own.begin(), own.end(), [&](const U &a, const U &b) {
+            return a.size + EPI_ADD * nparts_of(a) > b.size + EPI_ADD * nparts_of(b);
+        });
+        for (const U &u : own) {
+            const int np = nparts_of(u);
+            const Item it = {(u.mt << 24) | (u.nt << 8) | u.chunk, u.size, EPI_OWN + EPI_ADD * np,
+                             np > 0 ? (int)ready[(size_t)u.mt * nt + u.nt] + 3 : 0};
+            place(it, np > 0 ? 2 : 1);
+        }
+        std::vector<long long> load(G, 0);
+        std::vector<std::vector<int>> lists(G);
+        for (int c = 0; c < G; ++c) {
+            load[c] = finish(c, nullptr, 0);
+            for (const Item &it : lp[c]) lists[c].push_back(it.code);
+            for (const Item &it : lo0[c]) lists[c].push_back(it.code);
+            for (const Item &it : lo1[c]) lists[c].push_back(it.code);
+        }
+        if (getenv("JS_DEBUG_SCHED")) {
+            for (int c : {0, G / 2, G - 1}) {
+                fprintf(stderr, "layer %d ch %d cta %d load %lld:", l, ch, c, load[c]);
+                for (int v : lists[c]) fprintf(stderr, " (mt%d nt%d c%d kb%d)", v >> 24, (v >> 8) & 0xffff, v & 0xff, kb[(v >> 8) & 0xffff]);
+                fprintf(stderr, "\n");
+            }
+            long long mx = 0, mn = 1 << 30;
+            for (int c = 0; c < G; ++c) { mx = std::max(mx, load[c]); mn = std::min(mn, load[c]); }
+            fprintf(stderr, "layer %d: G %d units %zu+%zu load min %lld max %lld\n", l, G, part.size(), own.size(), mn, mx);
+        }
+        std::vector<int> off(G + 1, 0), flat;
+        for (int c = 0; c < G; ++c) { off[c] = (int)flat.size(); flat.insert(flat.end(), lists[c].begin(), lists[c].end()); }
+        off[G] = (int)flat.size();
+        auto up = [&](const std::vector<int> &h, const int **dst) -> bool {
+            void *q = nullptr;
+            if (cudaMalloc(&q, std::max<size_t>(h.size(), 1) * sizeof(int)) != cudaSuccess) return false;
+            mo->allocs.push_back(q);
+            if (!h.empty() && cudaMemcpy(q, h.data(), h.size() * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return false;
+            *dst = (const int *)q;
+            return true;
+        };
+        if (!up(slot_base, &t.lay[l].slot_base) || !up(off, &t.lay[l].sched_off) || !up(flat, &t.lay[l].sched)) return JS_ERR_CUDA;
+        t.lay[l].ch = ch;
+        t.lay[l].slots_per_mt = slots;
+        max_slots = std::max(max_slots, slots * MTmax);
+        part_floats = std::max(part_floats, (size_t)slots * MTmax * BM * bn);
+    }
+    {
+        void *q = nullptr;
+        if (cudaMalloc(&q, std::max<size_t>(part_floats, 4) * sizeof(float)) != cudaSuccess) return JS_ERR_CUDA;
+        mo->allocs.push_back(q);
+        t.partials = (float *)q;
+        t.n_pflags = std::max(max_slots, 1) * 4;
+        if (cudaMalloc(&q, (size_t)t.n_pflags * sizeof(unsigned)) != cudaSuccess) return JS_ERR_CUDA;
+        mo->allocs.push_back(q);
+        if (cudaMemset(q, 0, (size_t)t.n_pflags * sizeof(unsigned)) != cudaSuccess) return JS_ERR_CUDA;
+        t.pflags = (unsigned *)q;
     }
     void *pa = nullptr, *pw = nullptr;
     if (cudaMalloc(&pa, (L + 1) * sizeof(CUtensorMap)) != cudaSuccess) return JS_ERR_CUDA;
@@ -728,9 +1055,7 @@ int js_tc_prepare(js_model *mo)
         cudaGetLastError();      // not sticky: the CUDA-core kernels will serve this model
         return 0;
     }
-    int dev = 0, sms = 0, per_sm = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int per_sm = 0;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, made_tc_kernel, NTH, smem) != cudaSuccess || per_sm < 1)
         return 0;
     mo->tc_max_grid = sms;      // one CTA per SM: each owns all 512 TMEM columns
@@ -742,10 +1067,9 @@ int js_launch_made_tc(const js_model *mo, const RunArgs &r, cudaStream_t stream)
 {
     const MadeDev &v = mo->made;
     const TcDev &t = mo->tc;
-    const int MT = (r.batch + BM - 1) / BM;
-    int tiles = 1;
-    for (int l = 0; l <= v.L; ++l) tiles = std::max(tiles, t.lay[l].nt * MT);
-    const int grid = std::max(1, std::min(mo->tc_max_grid, tiles));
+    (void)r.batch;
+    const int grid = std::min(t.grid, mo->tc_max_grid);
+    if (grid != t.grid) return (int)cudaErrorInvalidConfiguration;     // the schedules need exactly t.grid CTAs
     void *args[3] = {(void *)&v, (void *)&t, (void *)&r};
     cudaError_t e = cudaLaunchCooperativeKernel((const void *)made_tc_kernel, dim3(grid), dim3(NTH), args,
                                                 t.smem_bytes, stream);

@@ -144,6 +144,19 @@ __device__ __forceinline__ uint32_t ld_u16_now(const uint8_t *p)
     return (uint32_t)v;
 }
 
+__device__ __forceinline__ float4 ld_nc_f4_now(const float *p)
+{
+    float4 v;
+    asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_u32_now(const uint8_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.global.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
 __device__ __forceinline__ void prefetch_l2(const void *p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 // 32 consecutive fp32 columns of this thread's TMEM lane

@@ -81,7 +81,10 @@ BIN = si.scaled(si.CONFIGS["made_784"], D=200, H=(192, 160), batch=70)        # 
 CAT = si.scaled(si.CONFIGS["made_cat"], D=24, H=(128, 96), batch=9)
 CHAIN = si.scaled(si.CONFIGS["made_4096"], D=256, H=(256, 256, 256, 256), batch=130, w_var_scale=4.0)
 
-CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN}
+# long K ranges with few tiles: the tensor-core kernels cut every tile's K loop into several work units
+SPLIT = si.scaled(si.CONFIGS["made_784"], D=1024, H=(1024, 1024), batch=130, w_var_scale=3.0)
+
+CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN, "split": SPLIT}
 # kernel path: 1 = CUDA-core kernels, 0 = tensor-core kernels (bf16 models only)
 COMBOS = [(n, 1) for n in CASES] + [(n, 0) for n in CASES if n != "tiny"]
 COMBO_IDS = [f"{n}-{'tc' if p == 0 else 'cc'}" for n, p in COMBOS]
@@ -159,7 +162,7 @@ def test_sequential_and_gauss_seidel(name, seq_skip):
 
 
 @pytest.mark.parametrize("name,blocks", [("tiny", (1, 4, 5, 16)), ("bin", (64, 30)), ("cat", (8, 5)),
-                                         ("chain", (32, 64))])
+                                         ("chain", (32, 64)), ("split", (256,))])
 @pytest.mark.parametrize("skip", [1, 0])
 def test_hybrids(name, blocks, skip):
     _skip_if_not_applicable(name)
