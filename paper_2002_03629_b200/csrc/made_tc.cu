@@ -907,7 +907,11 @@ int js_tc_prepare(js_model *mo)
         long long total_kb = 0;
         for (int x : kb) total_kb += (long long)x * MTmax;
         int ch = 1 << 20;                                              // enough tiles: no split
-        if ((long long)kb.size() * MTmax < 2LL * sms) {
+        int kb_longest = 1;
+        for (int x : kb) kb_longest = std::max(kb_longest, x);
+        // splitting pays only for long K loops: handing a partial sum over costs about as much
+        // as twenty K blocks of loading
+        if ((long long)kb.size() * MTmax < 2LL * sms && kb_longest >= 40) {
             // a CTA's fair share of the layer, but never less than half of the longest tile: every
             // extra chunk costs its owner a 64 KB read of partial sums
             int kb_max = 1;
