@@ -155,6 +155,23 @@ class ClockSampler:
 MODES = {"jacobi": 0, "gauss_seidel": 1, "gs_jacobi": 2, "jacobi_gs": 3}
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of per-rank timings (no-op without a process group).  Replicas exchange
+    nothing else: each rank samples its own batch."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_rate(samples_per_rank: int, steps: int, world: int, seconds: float) -> float:
+    """Samples per second of all replicas together, against the slowest rank's time."""
+    return samples_per_rank * steps * world / seconds
+
+
 def make_inputs(cfg):
     if cfg.kind == "conv":
         W, b = si.conv_weights(cfg)
@@ -310,10 +327,7 @@ def run_ours(args, cfg):
             seq[name + "_matches_jacobi"] = bool(torch.equal(out2, out))
         model.set_option(pkg.JS_OPT_SEQ_SKIP, 0)
 
-    if world > 1:
-        t = torch.tensor([total_ms, e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_s = float(t[0]), float(t[1])
+    total_ms, e2e_s = max_over_ranks([total_ms, e2e_s], device="cuda")
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -321,7 +335,7 @@ def run_ours(args, cfg):
 
     peaks = load_peaks()
     n_samples = cfg.batch * args.steps * world
-    value = n_samples / (total_ms / 1e3)
+    value = whole_job_rate(cfg.batch, args.steps, world, total_ms / 1e3)
     live = live_macs_per_sample(cfg)
     flops_per_launch = 2.0 * live * cfg.batch * stats.iterations
     ms_launch = total_ms / args.steps
