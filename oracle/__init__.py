@@ -40,7 +40,9 @@ _lib = None
 def lib():
     global _lib
     if _lib is None:
-        _lib = C.CDLL(build())
+        # ORACLE_LIB: a test plants mistakes in copies of the C source and points this at them,
+        # to show that the pins notice (tests/test_oracle_mutants.py)
+        _lib = C.CDLL(os.environ.get("ORACLE_LIB") or build())
         _lib.orc_made_create.restype = C.c_void_p
         _lib.orc_conv_create.restype = C.c_void_p
         _lib.orc_masked_weight.restype = C.POINTER(C.c_float)

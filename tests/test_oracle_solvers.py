@@ -173,6 +173,11 @@ def test_worked_examples_iteration_counts(kind, expected):
             assert m.jacobi_gs(noise[s], si.NOISE_LOGISTIC, 5)[1] == 4
         if kind == "independent":
             assert m.jacobi_gs(noise[s], si.NOISE_LOGISTIC, 5)[1] == 2
+            # Algorithm 3 starts every block from the initial guess: from a start that is wrong
+            # everywhere each of the M blocks needs one iteration to fix itself and one to confirm
+            # (an implementation that also updated later blocks early would need fewer)
+            wrong = (1 - xstar).astype(np.uint8)
+            assert m.gs_jacobi(noise[s], si.NOISE_LOGISTIC, 5, wrong)[1] == 2 * (T // 5)
 
 
 def test_critical_path_bound():
