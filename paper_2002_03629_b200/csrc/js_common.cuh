@@ -93,9 +93,10 @@ __device__ __forceinline__ bool grid_barrier(JsCtl *ctl, unsigned &epoch, unsign
     epoch += 1;
     int ok = 1;
     if (threadIdx.x == 0) {
-        __threadfence();
         const unsigned target = epoch * gridDim.x;
-        atomicAdd(&ctl->bar_count, 1u);
+        // arrive: a release at gpu scope (it also covers the other threads' writes, ordered before it
+        // by the __syncthreads above) with no value to wait for; the polls below are acquires
+        asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(&ctl->bar_count) : "memory");
         unsigned polls = 0;
         while (ld_acquire_u32(&ctl->bar_count) < target) {
             if (++polls > spin_limit || ld_volatile_i32(&ctl->abort) != 0) {
@@ -106,7 +107,6 @@ __device__ __forceinline__ bool grid_barrier(JsCtl *ctl, unsigned &epoch, unsign
             if (polls > 64) __nanosleep(64);
         }
         if (ok && ld_volatile_i32(&ctl->abort) != 0) ok = 0;
-        __threadfence();
     }
     return __syncthreads_and(ok) != 0;
 }
