@@ -79,15 +79,15 @@ def test_full_size_jacobi_and_hybrids(name):
 def test_full_size_jacobi_gs(name):
     p, cfg, orc, model, noise, d_noise, xstar = full_case(name)
     nk = cfg.noise_kind
-    B = cfg.blocks[0]
-    t0 = time.perf_counter()
-    x, it = run(p, cfg, model, d_noise, p.JS_JACOBI_GS, B)
-    print(f"{name}: jacobi-gs B={B} took {time.perf_counter() - t0:.2f} s, outer iters max {it.max()}")
-    audit = check_samples(orc, x, xstar, noise, nk)
-    ref = orc.map_batch(lambda i: orc.jacobi_gs(noise[i], nk, B)[1], 2, threads=2)
-    clean = [i for i in range(2) if i not in audit["excused_samples"]]
-    np.testing.assert_array_equal(it[clean], np.array(ref)[clean])
-    assert it.max() <= -(-cfg.D // B)
+    for B in cfg.blocks:
+        t0 = time.perf_counter()
+        x, it = run(p, cfg, model, d_noise, p.JS_JACOBI_GS, B)
+        print(f"{name}: jacobi-gs B={B} took {time.perf_counter() - t0:.2f} s, outer iters max {it.max()}")
+        audit = check_samples(orc, x, xstar, noise, nk)
+        ref = orc.map_batch(lambda i: orc.jacobi_gs(noise[i], nk, B)[1], 2, threads=2)
+        clean = [i for i in range(2) if i not in audit["excused_samples"]]
+        np.testing.assert_array_equal(it[clean], np.array(ref)[clean])
+        assert it.max() <= -(-cfg.D // B)
 
 
 @pytest.mark.parametrize("name", ["made_784", "made_4096", "made_cat"])

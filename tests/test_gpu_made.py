@@ -215,6 +215,41 @@ def test_compaction_changes_nothing_but_the_work():
     check_samples(c.orc, res[1][0], c.xstar, c.noise, c.nk)
 
 
+def test_tiny_model_brute_force_on_device():
+    """Config 1 on the device alone: logits of all 2^16 outcomes from js_forward_logits, the parallel
+    update of every outcome under each sample's noise, and exactly one fixed point - the sample that
+    jacobi_sample and sequential_sample return."""
+    if _path["v"] != 1:
+        pytest.skip("fp32 model: CUDA-core kernels")
+    p = pkg()
+    cfg = TINY
+    W, b = si.made_weights(cfg)
+    lut = si.made_lut(cfg)
+    noise = si.draw_noise(cfg)
+    D = cfg.D
+    big = p.Model.from_config(cfg, W, b, lut, max_batch=4096)
+    allx = ((np.arange(2 ** D)[:, None] >> np.arange(D)[None, :]) & 1).astype(np.uint8)
+    Z = np.empty((2 ** D, D), np.float32)
+    for s0 in range(0, 2 ** D, 4096):
+        logits = torch.empty((4096, D, 1), dtype=torch.float32, device="cuda")
+        assert p.js_forward_logits(big, torch.from_numpy(allx[s0:s0 + 4096]).cuda(), logits) == 0
+        Z[s0:s0 + 4096] = logits[:, :, 0].cpu().numpy()
+    P1 = (1.0 / (1.0 + np.exp(-Z.astype(np.float32)))).astype(np.float32)
+    d_noise = torch.from_numpy(noise).cuda()
+    out = torch.empty((cfg.batch, D), dtype=torch.uint8, device="cuda")
+    seq = torch.empty_like(out)
+    assert p.jacobi_sample(big, d_noise, cfg.noise_kind, None, p.JS_JACOBI, 0, 0, out, None) == 0
+    assert p.sequential_sample(big, d_noise, cfg.noise_kind, seq) == 0
+    got = out.cpu().numpy()
+    np.testing.assert_array_equal(got, seq.cpu().numpy())
+    for s in range(cfg.batch):
+        G = (noise[s][None, :] < P1).astype(np.uint8)
+        fixed = np.nonzero(np.all(G == allx, axis=1))[0]
+        assert len(fixed) == 1
+        np.testing.assert_array_equal(allx[fixed[0]], got[s])
+    big.close()
+
+
 def test_examples_of_section_4_on_device():
     """Markov chain (Example 3): T iterations; independent chain (Example 1): one plus the confirmation."""
     p = pkg()
