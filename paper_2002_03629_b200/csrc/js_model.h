@@ -19,7 +19,8 @@ struct TcLayer {
     int ch;
     int slots_per_mt;            // partial-sum slots per row tile = sum over nt of (chunks - 1)
     const int *slot_base;        // [nt] first slot of tile nt inside a row tile
-    const int *sched_off;        // [grid + 1] work units of CTA c: sched[sched_off[c] .. sched_off[c+1])
+    int n_sched;                 // schedules: one per number of live row tiles (1..n_sched), or a single one
+    const int *sched_off;        // [n_sched][grid + 1] work units of CTA c: sched[sched_off[c] .. sched_off[c+1])
     const int *sched;            // units packed as (row tile << 24) | (n tile << 8) | chunk
 };
 struct TcDev {
@@ -27,6 +28,8 @@ struct TcDev {
     const CUtensorMap *tmW;      // [L+1] masked weights W[l], box 64 x bn
     TcLayer lay[JS_MAXL + 1];
     int stage_bytes, n_stages, smem_bytes;
+    int ring_bytes, aux_bytes;   // shared memory: operand ring, then the epilogues' auxiliary buffer
+    int bin_bulk;                // binary output rows are 16-byte granular: moved by bulk copies
     int grid;                    // CTAs the schedules were built for (the launch uses exactly this)
     float *partials;             // [slot][columns/4][128 rows] float4: fp32 partial sums of non-owning chunks
     unsigned *pflags;            // [slot][4 row quadrants]: phase stamp once the partial is stored

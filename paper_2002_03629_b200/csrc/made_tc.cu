@@ -34,19 +34,24 @@ constexpr int BK = TC_BK;          // bf16 elements per K block
 constexpr int NTH = 192;
 constexpr int ACC_COLS = 256;      // TMEM columns per accumulator slot (two slots)
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int RING_BYTES = 160 * 1024;     // operand pipeline
 constexpr int STAGING_BYTES = 32 * 1024;   // epilogue transposition buffer, 8 KB per epilogue warp
 constexpr int MAX_STAGES = 6;
-constexpr int META_MAX_BYTES = 24 * 1024;   // shared memory left beside the ring for tile metadata
+// binary output tiles: per sample row 128 noise values and 128 symbols, rows padded by 16 bytes
+constexpr int BIN_NZ_ROW = 512 + 16, BIN_XS_ROW = 128 + 16;
+constexpr int BIN_NZ_BYTES = BM * BIN_NZ_ROW, BIN_XS_BYTES = BM * BIN_XS_ROW;
+// Shared memory after the 1 KB alignment slack: operand ring | auxiliary buffer | tile metadata.
+// The auxiliary buffer is the staging area of the hidden-layer epilogues and, in models with
+// binary outputs, also holds the noise and symbol rows of an output tile (never both at once).
+constexpr int SMEM_DYN_MAX = 227 * 1024 - 6 * 1024;      // what a CTA may ask for beside its static part
 
 enum { EPI_HIDDEN = 0, EPI_LOGITS = 1, EPI_BINARY = 2, EPI_CAT = 3 };
 
 struct TcShared {
     uint64_t full[MAX_STAGES], empty[MAX_STAGES], tfull[2], tempty[2];
+    uint64_t nzbar[4];             // per epilogue warp: bulk copies of a binary tile's noise and symbols
     uint32_t tmem_base;
     int off[JS_MAXL + 1];          // start of layer l's tile metadata inside `meta`
-    float bias_s[4][256];          // per epilogue warp: bias of the current tile's columns
-    int sb_s[4][32];               // per epilogue warp: row -> sample index of the current tile (-1: none)
+    alignas(16) float bias_s[4][256];   // per epilogue warp: bias of the current tile's columns (read as float4)
     int wcnt[NTH / 32];            // compaction: per-warp counts
     int cbase;                     // compaction: rows kept so far
 };
@@ -69,6 +74,7 @@ struct TcEngine {
     uint32_t sphase = 0;
     int acc = 0;
     uint32_t aphase = 0;
+    uint32_t nzphase = 0;
     bool dead = false;
     uint32_t tmem_base = 0;
     // working batch: rows [0, live) of the activation buffers hold samples perm[pcur][row]
@@ -77,7 +83,7 @@ struct TcEngine {
 
     __device__ TcEngine(const MadeDev &m_, const TcDev &t_, const RunArgs &r_, TcShared &sh_, uint8_t *ring_,
                         const int *meta_)
-        : m(m_), t(t_), r(r_), sh(sh_), ring(ring_), staging(ring_ + RING_BYTES), meta(meta_)
+        : m(m_), t(t_), r(r_), sh(sh_), ring(ring_), staging(ring_ + t_.ring_bytes), meta(meta_)
     {
         warp = threadIdx.x >> 5;
         lane = threadIdx.x & 31;
@@ -113,10 +119,27 @@ struct TcEngine {
     {
         const size_t n = (size_t)r.batch * m.T;
         __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
-        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-            const uint8_t v = src ? src[i] : (uint8_t)0;
-            if (r.x) r.x[i] = v;
-            a0[i] = __float2bfloat16_rn(m.lut[v]);
+        if (n % 16 == 0 && ((uintptr_t)src & 15u) == 0) {
+            // sixteen positions per step (the buffers are 16-byte aligned)
+            for (size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 16; i < n; i += (size_t)gridDim.x * blockDim.x * 16) {
+                const uint4 xv = src ? __ldcg(reinterpret_cast<const uint4 *>(src + i)) : make_uint4(0u, 0u, 0u, 0u);
+                if (r.x) *reinterpret_cast<uint4 *>(r.x + i) = xv;
+                const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+                uint32_t o[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    o[k] = pack_bf16x2(m.lut[(xw[k >> 1] >> (16 * (k & 1))) & 0xffu],
+                                       m.lut[(xw[k >> 1] >> (16 * (k & 1) + 8)) & 0xffu]);
+                uint4 *dst = reinterpret_cast<uint4 *>(a0 + i);
+                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+            }
+        } else {
+            for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+                const uint8_t v = src ? src[i] : (uint8_t)0;
+                if (r.x) r.x[i] = v;
+                a0[i] = __float2bfloat16_rn(m.lut[v]);
+            }
         }
         for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < (size_t)t.n_pflags;
              i += (size_t)gridDim.x * blockDim.x)
@@ -146,27 +169,32 @@ struct TcEngine {
         const int *chg = r.smp_changed + (size_t)parity * r.batch;
         if (threadIdx.x == 0) sh.cbase = 0;
         __syncthreads();
-        for (int base = 0; base < live; base += NTH) {
-            const int row = base + threadIdx.x;
-            int b = -1;
-            bool keep = false;
-            if (row < live) {
-                b = pc[row];
-                keep = ld_volatile_i32(&chg[b]) != 0;
+        // four rows per thread and round, their loads in flight together
+        for (int base = 0; base < live; base += 4 * NTH) {
+            int b[4];
+            bool keep[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int row = base + i * NTH + threadIdx.x;
+                b[i] = row < live ? __ldcg(&pc[row]) : -1;
             }
-            const unsigned bal = __ballot_sync(0xffffffffu, keep);
-            if (lane == 0) sh.wcnt[warp] = __popc(bal);
-            __syncthreads();
-            int off = sh.cbase;
-            for (int w2 = 0; w2 < warp; ++w2) off += sh.wcnt[w2];
-            if (keep) pn[off + __popc(bal & ((1u << lane) - 1u))] = b;
-            __syncthreads();
-            if (threadIdx.x == 0) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) keep[i] = b[i] >= 0 && ld_volatile_i32(&chg[b[i]]) != 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                if (base + i * NTH >= live) break;
+                const unsigned bal = __ballot_sync(0xffffffffu, keep[i]);
+                if (lane == 0) sh.wcnt[warp] = __popc(bal);
+                __syncthreads();
+                int off = sh.cbase;
+                for (int w2 = 0; w2 < warp; ++w2) off += sh.wcnt[w2];
+                if (keep[i]) pn[off + __popc(bal & ((1u << lane) - 1u))] = b[i];
                 int tot = 0;
                 for (int w2 = 0; w2 < NTH / 32; ++w2) tot += sh.wcnt[w2];
-                sh.cbase += tot;
+                __syncthreads();
+                if (threadIdx.x == 0) sh.cbase += tot;
+                __syncthreads();
             }
-            __syncthreads();
         }
         const int nlive = sh.cbase;
         __syncthreads();
@@ -176,10 +204,29 @@ struct TcEngine {
         if (blockIdx.x == 0 && threadIdx.x == 0) { r.ctl->compactions += 1; r.ctl->live = nlive; }
         __threadfence_block();
         __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
-        const size_t n = (size_t)live * m.T;
-        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-            const int row = (int)(i / m.T), d = (int)(i % m.T);
-            a0[i] = __float2bfloat16_rn(m.lut[r.x[(size_t)pn[row] * m.T + d]]);
+        if (m.T % 16 == 0) {
+            // sixteen positions per step: one 16-byte load of symbols, two 16-byte stores of encodings
+            const int per_row = m.T / 16;
+            const size_t n = (size_t)live * per_row;
+            for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+                const int row = (int)(i / per_row), d = (int)(i % per_row) * 16;
+                const uint4 xv = __ldcg(reinterpret_cast<const uint4 *>(r.x + (size_t)pn[row] * m.T + d));
+                const uint32_t xw[4] = {xv.x, xv.y, xv.z, xv.w};
+                uint32_t o[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    o[k] = pack_bf16x2(m.lut[(xw[k >> 1] >> (16 * (k & 1))) & 0xffu],
+                                       m.lut[(xw[k >> 1] >> (16 * (k & 1) + 8)) & 0xffu]);
+                uint4 *dst = reinterpret_cast<uint4 *>(a0 + (size_t)row * m.T + d);
+                dst[0] = make_uint4(o[0], o[1], o[2], o[3]);
+                dst[1] = make_uint4(o[4], o[5], o[6], o[7]);
+            }
+        } else {
+            const size_t n = (size_t)live * m.T;
+            for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+                const int row = (int)(i / m.T), d = (int)(i % m.T);
+                a0[i] = __float2bfloat16_rn(m.lut[r.x[(size_t)pn[row] * m.T + d]]);
+            }
         }
         return barrier() ? 1 : -1;
     }
@@ -235,16 +282,26 @@ struct TcEngine {
             u.nt = (v >> 8) & 0xffff;
             const int chunk = v & 0xff;
             if (u.mt >= MT || u.nt < nt_lo || u.nt >= nt_hi) continue;
+            // nc chunks of nearly equal length: the first `rem` of them hold one K block more
             const int kbe = kb_end_of(l, u.nt);
             const int nc = (kbe + ly.ch - 1) / ly.ch;
-            u.kb0 = chunk * ly.ch;
-            u.kb1 = min(kbe, u.kb0 + ly.ch);
+            const int base = kbe / nc, rem = kbe - base * nc;
+            u.kb0 = chunk * base + min(chunk, rem);
+            u.kb1 = u.kb0 + base + (chunk < rem ? 1 : 0);
             const bool owner = (chunk == nc - 1);
             u.nparts = owner ? nc - 1 : -1;
             u.slot = u.mt * ly.slots_per_mt + ly.slot_base[u.nt] + (owner ? 0 : chunk);
             return true;
         }
         return false;
+    }
+    // this CTA's unit list of layer l for a working batch of MT row tiles
+    __device__ void unit_list(int l, int MT, int &e, int &e_end) const
+    {
+        const TcLayer &ly = t.lay[l];
+        const int *so = ly.sched_off + (size_t)(ly.n_sched > 1 ? MT - 1 : 0) * (gridDim.x + 1);
+        e = so[blockIdx.x];
+        e_end = so[blockIdx.x + 1];
     }
 
     __device__ void producer(int l, int nt_lo, int nt_hi, int MT)
@@ -253,8 +310,8 @@ struct TcEngine {
         const CUtensorMap *ma = t.tmA + l, *mw = t.tmW + l;
         const uint32_t bytes = A_BYTES + ly.bn * BK * 2;
         trace(0);
-        int e = ly.sched_off[blockIdx.x];
-        const int e_end = ly.sched_off[blockIdx.x + 1];
+        int e, e_end;
+        unit_list(l, MT, e, e_end);
         Unit u;
         while (!dead && next_unit(l, e, e_end, nt_lo, nt_hi, MT, u)) {
             issued++;
@@ -272,8 +329,8 @@ struct TcEngine {
     {
         const TcLayer &ly = t.lay[l];
         const uint32_t idesc = instr_desc_bf16(ly.bn);
-        int e = ly.sched_off[blockIdx.x];
-        const int e_end = ly.sched_off[blockIdx.x + 1];
+        int e, e_end;
+        unit_list(l, MT, e, e_end);
         Unit u;
         bool first = true;
         while (!dead && next_unit(l, e, e_end, nt_lo, nt_hi, MT, u)) {
@@ -509,119 +566,142 @@ struct TcEngine {
         if (ld_volatile_i32(f) == 0) *f = 1;
     }
 
-    // start this warp's rows of noise and symbols of a binary output tile towards L2 while the
-    // accumulator is still being computed (lane = row)
-    __device__ void bin_prefetch(int sample, int n0)
-    {
-        if (sample < 0 || n0 >= m.T) return;
-        const size_t at = (size_t)sample * m.T + n0;
-        const int ncols = min(128, m.T - n0);
-        for (int c = 0; c < ncols; c += 32) prefetch_l2(r.noise + at + c);
-        prefetch_l2(r.x + at);
-    }
+    // ---- binary output layer (128 positions per tile), thread = one sample row of the tile.
+    // The row's noise (512 bytes) and current symbols (128 bytes) are brought into shared memory by
+    // bulk copies that are issued before the accumulator is waited for, so they travel while the
+    // K loop still runs; rows are padded by 16 bytes, which makes the row-per-lane 16-byte accesses
+    // conflict-free.  The new symbols replace the old ones in place, the new encodings (bf16)
+    // overwrite the part of the noise row that has been consumed, and a row in which something
+    // changed goes back to global memory as two bulk stores.
+    __device__ uint8_t *nz_row() const { return staging + (size_t)((warp & 3) * 32 + lane) * BIN_NZ_ROW; }
+    __device__ uint8_t *xs_row() const { return staging + BIN_NZ_BYTES + (size_t)((warp & 3) * 32 + lane) * BIN_XS_ROW; }
 
-    // binary output layer: 128 positions per tile in two halves of 64: threshold the logit against
-    // the fixed noise, compare with the current symbol, commit symbol and encoding, note changes
-    // noise and current symbols of eight row pairs (rows (g+j)*2 + rsel) at this lane's four positions
-    struct BinRows {
-        float4 nz[8];
-        uint32_t xo[8];
-        int sb[8];
-    };
-    __device__ void bin_load_rows(BinRows &in, const int *sbs, int g, int d, bool any_in) const
+    __device__ void bin_fetch_rows(int smp, int n0, int ncols)
     {
-        const int rsel = lane >> 4;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int rl = (g + j) * 2 + rsel;
-            in.sb[j] = sbs[rl];
-            in.nz[j] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-            in.xo[j] = 0;
-            if (in.sb[j] >= 0 && any_in) {
-                const size_t at = (size_t)in.sb[j] * m.T + d;
-                in.nz[j] = ld_nc_f4_now(r.noise + at);      // issued here, not at first use
-                in.xo[j] = ld_u32_now(r.x + at);
+        const int q = warp & 3;
+        bulk_wait_read();                     // this thread's earlier bulk stores no longer read the rows
+        __syncwarp();
+        if (t.bin_bulk) {
+            const uint32_t bytes = smp >= 0 ? (uint32_t)ncols * 5u : 0u;
+            const uint32_t tot = __reduce_add_sync(0xffffffffu, bytes);
+            if (lane == 0) mbar_expect_tx(&sh.nzbar[q], tot);
+            __syncwarp();
+            if (smp >= 0) {
+                const size_t at = (size_t)smp * m.T + n0;
+                bulk_load(smem_u32(nz_row()), r.noise + at, (uint32_t)ncols * 4u, &sh.nzbar[q]);
+                bulk_load(smem_u32(xs_row()), r.x + at, (uint32_t)ncols, &sh.nzbar[q]);
+            }
+        } else if (smp >= 0) {
+            // widths that are not multiples of 16: plain loads (8 positions at a time)
+            const size_t at = (size_t)smp * m.T + n0;
+            uint8_t *nz = nz_row(), *xs = xs_row();
+            for (int c = 0; c < ncols; c += 8) {
+                const float4 v0 = ld_nc_f4_now(r.noise + at + c), v1 = ld_nc_f4_now(r.noise + at + c + 4);
+                const uint2 xv = __ldcg(reinterpret_cast<const uint2 *>(r.x + at + c));
+                *reinterpret_cast<float4 *>(nz + c * 4) = v0;
+                *reinterpret_cast<float4 *>(nz + c * 4 + 16) = v1;
+                *reinterpret_cast<uint2 *>(xs + c) = xv;
             }
         }
     }
-    __device__ void bin_decide_rows(const BinRows &in, int g, int mt, int d, unsigned inm, const float (&bias4)[4],
-                                    unsigned &chmask, int &lfirst)
-    {
-        uint8_t *stg = my_staging();
-        const int q = warp & 3, ch = lane & 15, rsel = lane >> 4, T_ = m.T;
-        __nv_bfloat16 *a0 = (__nv_bfloat16 *)m.a[0];
-        const float lut0 = m.lut[0], lut1 = m.lut[1];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const int rl = (g + j) * 2 + rsel;
-            const float4 v = *reinterpret_cast<const float4 *>(stg + rl * 256 + ((ch ^ (rl & 15)) << 4));
-            bool changed = false;
-            if (in.sb[j] >= 0 && inm != 0u) {
-                const float z[4] = {v.x + bias4[0], v.y + bias4[1], v.z + bias4[2], v.w + bias4[3]};
-                const float e[4] = {in.nz[j].x, in.nz[j].y, in.nz[j].z, in.nz[j].w};
-                uint32_t xn = 0;
-                float enc[4];
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint32_t o = (in.xo[j] >> (8 * c)) & 0xffu;
-                    const uint32_t nv = ((inm >> c) & 1u) ? (uint32_t)js_sample_binary(r.nk, z[c], e[c]) : o;
-                    if (nv != o && d + c < lfirst) lfirst = d + c;
-                    xn |= nv << (8 * c);
-                    enc[c] = nv ? lut1 : lut0;
-                }
-                changed = xn != in.xo[j];
-                if (changed) {
-                    *reinterpret_cast<uint32_t *>(r.x + (size_t)in.sb[j] * T_ + d) = xn;
-                    const int row = mt * BM + q * 32 + rl;
-                    *reinterpret_cast<uint2 *>(a0 + (size_t)row * T_ + d) =
-                        make_uint2(pack_bf16x2(enc[0], enc[1]), pack_bf16x2(enc[2], enc[3]));
-                }
-            }
-            // bit = row of the warp; no warp vote here, so that the eight iterations can overlap
-            if (changed) chmask |= 1u << rl;
-        }
-    }
 
-    // binary output layer: 128 positions per tile in two halves of 64: threshold the logit against
-    // the fixed noise, compare with the current symbol, commit symbol and encoding, note changes.
-    // The loads of a half's first sixteen rows are issued before the accumulator is staged, those of
-    // the other sixteen before the first ones are used, so that little memory latency stays exposed.
-    __device__ void epi_binary_tile(const Win &w, int mt, int n0, uint32_t tbase, bool flag, int parity,
-                                    bool &wany, int &wfirst)
+    __device__ bool epi_binary_tile(const Win &w, int smp, int rw, int n0, int ncols, uint32_t tbase, bool flag,
+                                    int parity, bool &wany, int &wfirst)
     {
         const float *bs = sh.bias_s[warp - 2];
-        const int *sbs = sh.sb_s[warp - 2];
-        const int T_ = m.T, ch = lane & 15;
-        unsigned chmask = 0;           // rows in which this lane changed something (bit = row of the warp)
-        int lfirst = INT_MAX;          // this lane's smallest changed position
+        uint8_t *nz = nz_row(), *xs = xs_row();
+        const float lut0 = m.lut[0], lut1 = m.lut[1];
+        const int nk = r.nk;
+        // columns [clo, chi) of the tile are sampled; the others keep their symbol
+        const int clo = max(w.plo - n0, 0), chi = min(min(w.phi, m.T) - n0, ncols);
+        if (t.bin_bulk) {
+            if (!mbar_wait(&sh.nzbar[warp & 3], nzphase, r.ctl)) return false;
+            nzphase ^= 1u;
+        }
+        uint32_t diff_any = 0;
+        int first = INT_MAX;
+        const bool tr = (warp == 2 && lane == 0);
+        if (tr) trace(6);
 #pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
-            const int cb = half * 64 + ch * 4;
-            const int d = n0 + cb;                               // this lane's four positions d..d+3
-            unsigned inm = 0;                                    // which of them are inside the window
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (d + j >= w.plo && d + j < w.phi && d + j < T_) inm |= 1u << j;
-            const float bias4[4] = {bs[cb], bs[cb + 1], bs[cb + 2], bs[cb + 3]};
-            BinRows ra, rb;
-            const bool tr = (warp == 2 && lane == 0);
-            if (tr) trace(6 + 3 * half);
-            bin_load_rows(ra, sbs, 0, d, inm != 0u);
-            stage_half(tbase, half);
-            if (half == 1) release_acc(); else __syncwarp();
-            if (tr) trace(7 + 3 * half);
-            bin_load_rows(rb, sbs, 8, d, inm != 0u);
-            bin_decide_rows(ra, 0, mt, d, inm, bias4, chmask, lfirst);
-            if (tr) trace(8 + 3 * half);
-            bin_decide_rows(rb, 8, mt, d, inm, bias4, chmask, lfirst);
+        for (int c0 = 0; c0 < BM; c0 += 32) {
+            uint32_t ra[32];
             __syncwarp();
+            tmem_ld32_issue(tbase + (uint32_t)c0, ra);
+            tmem_wait_ld();
+            if (c0 == BM - 32) release_acc();
+            if (cur_parts > 0) add_partials(ra, c0);
+            if (smp >= 0 && c0 < ncols) {
+                // everything the 32 columns need is read before anything is written: the stores below
+                // go to the same rows, and a load may not overtake a store it might alias
+                float4 e4[8], b4[8];
+                uint4 xo4[2];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) e4[i] = *reinterpret_cast<const float4 *>(nz + (c0 + i * 4) * 4);
+#pragma unroll
+                for (int i = 0; i < 2; ++i) xo4[i] = *reinterpret_cast<const uint4 *>(xs + c0 + i * 16);
+#pragma unroll
+                for (int i = 0; i < 8; ++i) b4[i] = *reinterpret_cast<const float4 *>(bs + c0 + i * 4);
+                uint32_t xn[8];
+                uint2 en[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int c = c0 + i * 4;
+                    const uint32_t xw = (i & 3) == 0 ? xo4[i >> 2].x : (i & 3) == 1 ? xo4[i >> 2].y
+                                      : (i & 3) == 2 ? xo4[i >> 2].z : xo4[i >> 2].w;
+                    const float e[4] = {e4[i].x, e4[i].y, e4[i].z, e4[i].w};
+                    const float bb[4] = {b4[i].x, b4[i].y, b4[i].z, b4[i].w};
+                    uint32_t nw = 0;
+                    float enc[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        const uint32_t o = (xw >> (8 * k)) & 0xffu;
+                        const float z = __uint_as_float(ra[i * 4 + k]) + bb[k];
+                        const bool in = (unsigned)(c + k - clo) < (unsigned)(chi - clo);
+                        const uint32_t nv = in ? (uint32_t)js_sample_binary(nk, z, e[k]) : o;
+                        nw |= nv << (8 * k);
+                        enc[k] = nv ? lut1 : lut0;
+                    }
+                    const uint32_t df = nw ^ xw;
+                    if (df != 0u && first == INT_MAX) first = n0 + c + ((__ffs((int)df) - 1) >> 3);
+                    diff_any |= df;
+                    xn[i] = nw;
+                    en[i] = make_uint2(pack_bf16x2(enc[0], enc[1]), pack_bf16x2(enc[2], enc[3]));
+                }
+                // new symbols in place; encodings over noise that has been consumed (bytes [2c, 2c+8)
+                // of the row lie below the noise of column c+4 and beyond)
+                *reinterpret_cast<uint4 *>(xs + c0) = make_uint4(xn[0], xn[1], xn[2], xn[3]);
+                *reinterpret_cast<uint4 *>(xs + c0 + 16) = make_uint4(xn[4], xn[5], xn[6], xn[7]);
+#pragma unroll
+                for (int i = 0; i < 8; i += 2)
+                    *reinterpret_cast<uint4 *>(nz + (c0 + i * 4) * 2) = make_uint4(en[i].x, en[i].y, en[i + 1].x, en[i + 1].y);
+            }
         }
-        chmask = __reduce_or_sync(0xffffffffu, chmask);           // rows changed by any lane
-        if (flag && chmask != 0u) {
-            if (((chmask >> lane) & 1u) && sbs[lane] >= 0) raise_flag(parity, sbs[lane]);      // lane = row
-            wany = true;
-            wfirst = min(wfirst, __reduce_min_sync(0xffffffffu, lfirst));
+        __syncwarp();
+        if (tr) trace(7);
+        const bool changed = diff_any != 0u;
+        if (t.bin_bulk) {
+            fence_proxy_async_smem();         // the rows were written through the generic proxy
+            if (changed) {
+                bulk_store(r.x + (size_t)smp * m.T + n0, smem_u32(xs), (uint32_t)ncols);
+                bulk_store((__nv_bfloat16 *)m.a[0] + (size_t)rw * m.T + n0, smem_u32(nz), (uint32_t)ncols * 2u);
+                bulk_commit();
+            }
+        } else if (changed) {
+            uint8_t *xg = r.x + (size_t)smp * m.T + n0;
+            __nv_bfloat16 *ag = (__nv_bfloat16 *)m.a[0] + (size_t)rw * m.T + n0;
+            for (int c = 0; c < ncols; c += 8) {
+                *reinterpret_cast<uint2 *>(xg + c) = *reinterpret_cast<const uint2 *>(xs + c);
+                *reinterpret_cast<uint4 *>(ag + c) = *reinterpret_cast<const uint4 *>(nz + c * 2);
+            }
         }
+        if (flag) {
+            if (changed) raise_flag(parity, smp);
+            if (__any_sync(0xffffffffu, changed)) {
+                wany = true;
+                wfirst = min(wfirst, __reduce_min_sync(0xffffffffu, first));
+            }
+        }
+        return true;
     }
 
     __device__ void epilogue(int l, int kind, const Win &w, bool flag, int parity, float *zout, int nt_lo,
@@ -631,20 +711,26 @@ struct TcEngine {
         const int q = warp & 3;
         bool any_changed = false;
         int first = INT_MAX;
-        int e = ly.sched_off[blockIdx.x];
-        const int e_end = ly.sched_off[blockIdx.x + 1];
+        int e, e_end;
+        unit_list(l, MT, e, e_end);
         Unit u;
         while (!dead && next_unit(l, e, e_end, nt_lo, nt_hi, MT, u)) {
             const int nt = u.nt, mt = u.mt;
             const bool owner = u.nparts >= 0;
             if (owner && (kind == EPI_HIDDEN || kind == EPI_BINARY)) load_bias_tile(l, nt * ly.bn, ly.bn);
+            int bsmp = -1, bcols = 0;
             if (owner && kind == EPI_BINARY) {
                 const int rw = mt * BM + q * 32 + lane;
-                const int smp = rw < live ? perm_cur()[rw] : -1;
-                __syncwarp();
-                sh.sb_s[warp - 2][lane] = smp;
-                __syncwarp();
-                bin_prefetch(smp, nt * ly.bn);              // in flight while the tile is still being computed
+                bsmp = rw < live ? perm_cur()[rw] : -1;
+                bcols = min(BM, m.T - nt * ly.bn);
+                bin_fetch_rows(bsmp, nt * ly.bn, bcols);     // in flight while the tile is still being computed
+            }
+            if (owner) {
+                cur_parts = u.nparts;
+                cur_pbase = t.partials + (size_t)u.slot * tile_floats(l);
+                cur_tile_floats = tile_floats(l);
+                // partial sums do not depend on this CTA's accumulator: wait for them first
+                if (cur_parts > 0 && !wait_partials(u.slot, cur_parts)) { dead = true; break; }
             }
             if (!mbar_wait(&sh.tfull[acc], aphase, r.ctl)) { dead = true; break; }
             tc_fence_after();
@@ -657,16 +743,12 @@ struct TcEngine {
                 advance_acc();
                 continue;
             }
-            cur_parts = u.nparts;
-            cur_pbase = t.partials + (size_t)u.slot * tile_floats(l);
-            cur_tile_floats = tile_floats(l);
-            if (cur_parts > 0 && !wait_partials(u.slot, cur_parts)) { dead = true; break; }
             if (kind == EPI_HIDDEN) {
                 epi_hidden_tile(l, mt, n0, tbase);
             } else if (kind == EPI_BINARY) {
                 bool wany = false;
                 int wfirst = INT_MAX;
-                epi_binary_tile(w, mt, n0, tbase, flag, parity, wany, wfirst);
+                if (!epi_binary_tile(w, bsmp, row, n0, bcols, tbase, flag, parity, wany, wfirst)) { dead = true; break; }
                 if (wany) { any_changed = true; first = min(first, wfirst); }
             } else {
                 float best = -INFINITY;
@@ -705,6 +787,7 @@ struct TcEngine {
             }
             advance_acc();
         }
+        bulk_wait_all();          // bulk stores of this phase are complete before the grid barrier
         if (warp == 2 && lane == 0) trace(4);
         if (flag) {
             const bool wany = __any_sync(0xffffffffu, any_changed);
@@ -762,16 +845,19 @@ made_tc_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ TcDev 
     uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
 
     const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0 && r.trace != nullptr && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1))
+        r.trace[((size_t)(blockIdx.x == 0 ? 0 : 1) * JS_TRACE_PHASES) * JS_TRACE_SLOTS + 2] = global_ns();   // kernel entry
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 4); }
+        for (int a = 0; a < 4; ++a) mbar_init(&sh.nzbar[a], 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
     if (warp == 1) tmem_alloc(&sh.tmem_base, 512);
     // tile metadata of every layer into shared memory (the range searches and the K-loop bounds
     // would otherwise be chains of dependent global loads in every phase)
-    int *meta = reinterpret_cast<int *>(ring + RING_BYTES + STAGING_BYTES);
+    int *meta = reinterpret_cast<int *>(ring + t.ring_bytes + t.aux_bytes);
     {
         int off = 0;
         for (int l = 0; l <= m.L; ++l) {
@@ -791,8 +877,10 @@ made_tc_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ TcDev 
 
     TcEngine e(m, t, r, sh, ring, meta);
     e.tmem_base = sh.tmem_base;
+    if (threadIdx.x == 0) e.trace(0);
     DriverResult res = made_driver(e, m.T, r);
     if (e.dead) res.alive = false;
+    if (threadIdx.x == 0) { e.phase_no = 0; e.trace(1); }
 
     // leave: let copies still in flight land (only possible after an aborted wait), free TMEM
     tc_fence_before();
@@ -858,8 +946,15 @@ int js_tc_prepare(js_model *mo)
     const int L = v.L;
     bool wide = (v.C == 256);
     t.stage_bytes = A_BYTES + (wide ? 256 : 128) * BK * 2;
-    t.n_stages = RING_BYTES / t.stage_bytes;
-    if (t.n_stages > MAX_STAGES) t.n_stages = MAX_STAGES;
+    int meta_ints = 0;
+    for (int l = 0; l <= L; ++l) meta_ints += 3 * ((v.n[l + 1] + ((l == L && wide) ? 256 : 128) - 1) / ((l == L && wide) ? 256 : 128));
+    const int meta_bytes = (meta_ints * 4 + 127) & ~127;
+    t.aux_bytes = wide ? STAGING_BYTES : std::max(STAGING_BYTES, BIN_NZ_BYTES + BIN_XS_BYTES);
+    t.bin_bulk = (!wide && v.T % 16 == 0) ? 1 : 0;
+    t.n_stages = (SMEM_DYN_MAX - 1024 - t.aux_bytes - meta_bytes) / t.stage_bytes;
+    if (t.n_stages > (wide ? 3 : 4)) t.n_stages = wide ? 3 : 4;
+    if (t.n_stages < 2) return 0;
+    t.ring_bytes = t.n_stages * t.stage_bytes;
     std::vector<CUtensorMap> mapsA(L + 1), mapsW(L + 1);
     std::vector<std::vector<int>> kb_all(L + 1);
     for (int l = 0; l <= L; ++l) {
@@ -910,14 +1005,13 @@ int js_tc_prepare(js_model *mo)
         int kb_longest = 1;
         for (int x : kb) kb_longest = std::max(kb_longest, x);
         // splitting pays only for long K loops: handing a partial sum over costs about as much
-        // as twenty K blocks of loading
-        if ((long long)kb.size() * MTmax < 2LL * sms && kb_longest >= 40) {
-            // a CTA's fair share of the layer, but never less than half of the longest tile: every
-            // extra chunk costs its owner a 64 KB read of partial sums
-            int kb_max = 1;
-            for (int x : kb) kb_max = std::max(kb_max, x);
-            ch = (int)std::max<long long>(std::max<long long>(4, (kb_max + 1) / 2), (total_kb + sms - 1) / sms);
-        }
+        // as ten K blocks of loading
+        // The chain  longest K loop -> hand-over -> owner's epilogue  is what a phase has to wait for,
+        // so hidden layers cut their longest tiles into about three chunks (measured best on 64 K
+        // blocks: chunks of 20; 32 and 12 are each 12 % slower); the output layer, whose epilogue is
+        // the long part, into two.
+        if ((long long)kb.size() * MTmax < 2LL * sms && kb_longest >= 40)
+            ch = std::max(4, l < L ? (kb_longest * 5 + 15) / 16 : (kb_longest + 1) / 2);
         chs[l] = ch;
         long long units = 0;
         for (int x : kb) units += (long long)((x + ch - 1) / ch) * MTmax;
@@ -926,94 +1020,100 @@ int js_tc_prepare(js_model *mo)
     t.grid = G;
     size_t part_floats = 0;
     int max_slots = 0;
+    // One schedule per size of the working batch (compaction shrinks it), as long as that is a
+    // handful; the chunks themselves never depend on it, only who computes them.
+    const int n_sched = MTmax <= 16 ? MTmax : 1;
     for (int l = 0; l <= L; ++l) {
         const std::vector<int> &kb = kb_all[l];
         const int ch = chs[l], nt = (int)kb.size(), bn = t.lay[l].bn;
         std::vector<int> slot_base(nt);
         int slots = 0;
         for (int i = 0; i < nt; ++i) { slot_base[i] = slots; slots += (kb[i] + ch - 1) / ch - 1; }
-        // units: non-owning chunks first (all of size ch), then owners by decreasing size
-        struct U { int mt, nt, chunk, size; };
-        std::vector<U> part, own;
-        for (int mt = 0; mt < MTmax; ++mt)
-            for (int i = 0; i < nt; ++i) {
-                const int nc = (kb[i] + ch - 1) / ch;
-                for (int c = 0; c + 1 < nc; ++c) part.push_back({mt, i, c, ch});
-                own.push_back({mt, i, nc - 1, kb[i] - ch * (nc - 1)});
-            }
-        // List scheduling on a small model of a CTA, in units of one K block's load time: the K
-        // loops of a CTA's units run back to back; a unit's epilogue starts when its K loop is
-        // done, the previous epilogue is done and (for an owner) the tile's partial sums have been
-        // stored.  Units are taken longest first and put where the CTA finishes earliest.  Inside
-        // a CTA: partial chunks first (owners elsewhere wait for them), then owners that wait for
-        // nobody, then owners that add partial sums.
-        const int EPI_PART = 7, EPI_OWN = (l == L ? 24 : 10), EPI_ADD = 7;
-        auto nparts_of = [&](const U &u) { return (kb[u.nt] + ch - 1) / ch - 1; };
-        struct Item { int code, size, epi, ready; };
-        std::vector<std::vector<Item>> lp(G), lo0(G), lo1(G);
-        auto finish = [&](int c, const Item *extra, int where) {
-            long long M = 2, E = 0;
-            auto run = [&](const Item &it) {
-                M += it.size;
-                const long long start = std::max<long long>(std::max(M, E), it.ready);
-                E = start + it.epi;
+        auto chunk_len = [&](int i, int c) {
+            const int nc = (kb[i] + ch - 1) / ch, base = kb[i] / nc, rem = kb[i] - base * nc;
+            return base + (c < rem ? 1 : 0);
+        };
+        auto nparts_of_tile = [&](int i) { return (kb[i] + ch - 1) / ch - 1; };
+        std::vector<int> off, flat;
+        for (int si = 0; si < n_sched; ++si) {
+            const int MT = n_sched > 1 ? si + 1 : MTmax;
+            // units: non-owning chunks first, then owners
+            struct U { int mt, nt, chunk, size; };
+            std::vector<U> part, own;
+            for (int mt = 0; mt < MT; ++mt)
+                for (int i = 0; i < nt; ++i) {
+                    const int nc = nparts_of_tile(i) + 1;
+                    for (int c = 0; c + 1 < nc; ++c) part.push_back({mt, i, c, chunk_len(i, c)});
+                    own.push_back({mt, i, nc - 1, chunk_len(i, nc - 1)});
+                }
+            // List scheduling on a small model of a CTA, in units of one K block's load time
+            // (about 0.35 us): the K loops of a CTA's units run back to back; a unit's epilogue
+            // starts when its K loop is done, the previous epilogue is done and (for an owner) the
+            // tile's partial sums have been stored.  Units are taken longest first and put where
+            // the CTA finishes earliest.  Inside a CTA: partial chunks first (owners elsewhere
+            // wait for them), then owners that wait for nobody, then owners that add partial sums.
+            const int FILL = 6, EPI_PART = 5, EPI_OWN = (l == L ? (bn == 256 ? 24 : 9) : 4), EPI_ADD = 8;
+            struct Item { int code, size, epi, ready; };
+            std::vector<std::vector<Item>> lp(G), lo0(G), lo1(G);
+            auto finish = [&](int c, const Item *extra, int where) {
+                long long M = FILL, E = 0;
+                auto run = [&](const Item &it) {
+                    M += it.size;
+                    const long long start = std::max<long long>(std::max(M, E), it.ready);
+                    E = start + it.epi;
+                };
+                for (const Item &it : lp[c]) run(it);
+                if (extra && where == 0) run(*extra);
+                for (const Item &it : lo0[c]) run(it);
+                if (extra && where == 1) run(*extra);
+                for (const Item &it : lo1[c]) run(it);
+                if (extra && where == 2) run(*extra);
+                return E;
             };
-            for (const Item &it : lp[c]) run(it);
-            if (extra && where == 0) run(*extra);
-            for (const Item &it : lo0[c]) run(it);
-            if (extra && where == 1) run(*extra);
-            for (const Item &it : lo1[c]) run(it);
-            if (extra && where == 2) run(*extra);
-            return E;
-        };
-        auto place = [&](const Item &it, int where) {
-            int best = 0;
-            long long bt = -1;
+            auto place = [&](const Item &it, int where) {
+                int best = 0;
+                long long bt = -1;
+                for (int c = 0; c < G; ++c) {
+                    const long long f = finish(c, &it, where);
+                    if (bt < 0 || f < bt) { bt = f; best = c; }
+                }
+                (where == 0 ? lp : where == 1 ? lo0 : lo1)[best].push_back(it);
+                return best;
+            };
+            std::stable_sort(part.begin(), part.end(), [](const U &a, const U &b) { return a.size > b.size; });
+            std::vector<long long> ready((size_t)MT * nt, 0);          // when a tile's partial sums are all stored
+            for (const U &u : part) {
+                const Item it = {(u.mt << 24) | (u.nt << 8) | u.chunk, u.size, EPI_PART, 0};
+                const int c = place(it, 0);
+                long long M = FILL, E = 0;                             // completion of this chunk in its CTA
+                for (const Item &x : lp[c]) { M += x.size; E = std::max(M, E) + x.epi; }
+                ready[(size_t)u.mt * nt + u.nt] = std::max(ready[(size_t)u.mt * nt + u.nt], E);
+            }
+            std::stable_sort(own.begin(), own.end(), [&](const U &a, const U &b) {
+                return a.size + EPI_ADD * nparts_of_tile(a.nt) > b.size + EPI_ADD * nparts_of_tile(b.nt);
+            });
+            for (const U &u : own) {
+                const int np = nparts_of_tile(u.nt);
+                const Item it = {(u.mt << 24) | (u.nt << 8) | u.chunk, u.size, EPI_OWN + EPI_ADD * np,
+                                 np > 0 ? (int)ready[(size_t)u.mt * nt + u.nt] + 3 : 0};
+                place(it, np > 0 ? 2 : 1);
+            }
+            std::vector<long long> load(G, 0);
             for (int c = 0; c < G; ++c) {
-                const long long f = finish(c, &it, where);
-                if (bt < 0 || f < bt) { bt = f; best = c; }
+                load[c] = finish(c, nullptr, 0);
+                off.push_back((int)flat.size());
+                for (const Item &it : lp[c]) flat.push_back(it.code);
+                for (const Item &it : lo0[c]) flat.push_back(it.code);
+                for (const Item &it : lo1[c]) flat.push_back(it.code);
             }
-            (where == 0 ? lp : where == 1 ? lo0 : lo1)[best].push_back(it);
-            return best;
-        };
-        std::vector<long long> ready((size_t)MTmax * nt, 0);          // when a tile's partial sums are all stored
-        for (const U &u : part) {
-            const Item it = {(u.mt << 24) | (u.nt << 8) | u.chunk, u.size, EPI_PART, 0};
-            const int c = place(it, 0);
-            long long M = 2, E = 0;                                    // completion of this chunk in its CTA
-            for (const Item &x : lp[c]) { M += x.size; E = std::max(M, E) + x.epi; }
-            ready[(size_t)u.mt * nt + u.nt] = std::max(ready[(size_t)u.mt * nt + u.nt], E);
-        }
-        std::stable_sort(own.begin(), own.end(), [&](const U &a, const U &b) {
-            return a.size + EPI_ADD * nparts_of(a) > b.size + EPI_ADD * nparts_of(b);
-        });
-        for (const U &u : own) {
-            const int np = nparts_of(u);
-            const Item it = {(u.mt << 24) | (u.nt << 8) | u.chunk, u.size, EPI_OWN + EPI_ADD * np,
-                             np > 0 ? (int)ready[(size_t)u.mt * nt + u.nt] + 3 : 0};
-            place(it, np > 0 ? 2 : 1);
-        }
-        std::vector<long long> load(G, 0);
-        std::vector<std::vector<int>> lists(G);
-        for (int c = 0; c < G; ++c) {
-            load[c] = finish(c, nullptr, 0);
-            for (const Item &it : lp[c]) lists[c].push_back(it.code);
-            for (const Item &it : lo0[c]) lists[c].push_back(it.code);
-            for (const Item &it : lo1[c]) lists[c].push_back(it.code);
-        }
-        if (getenv("JS_DEBUG_SCHED")) {
-            for (int c : {0, G / 2, G - 1}) {
-                fprintf(stderr, "layer %d ch %d cta %d load %lld:", l, ch, c, load[c]);
-                for (int v : lists[c]) fprintf(stderr, " (mt%d nt%d c%d kb%d)", v >> 24, (v >> 8) & 0xffff, v & 0xff, kb[(v >> 8) & 0xffff]);
-                fprintf(stderr, "\n");
+            off.push_back((int)flat.size());
+            if (getenv("JS_DEBUG_SCHED")) {
+                long long mx = 0, mn = 1 << 30;
+                for (int c = 0; c < G; ++c) { mx = std::max(mx, load[c]); mn = std::min(mn, load[c]); }
+                fprintf(stderr, "layer %d MT %d ch %d: G %d units %zu+%zu modelled finish min %lld max %lld\n", l, MT, ch, G,
+                        part.size(), own.size(), mn, mx);
             }
-            long long mx = 0, mn = 1 << 30;
-            for (int c = 0; c < G; ++c) { mx = std::max(mx, load[c]); mn = std::min(mn, load[c]); }
-            fprintf(stderr, "layer %d: G %d units %zu+%zu load min %lld max %lld\n", l, G, part.size(), own.size(), mn, mx);
         }
-        std::vector<int> off(G + 1, 0), flat;
-        for (int c = 0; c < G; ++c) { off[c] = (int)flat.size(); flat.insert(flat.end(), lists[c].begin(), lists[c].end()); }
-        off[G] = (int)flat.size();
         auto up = [&](const std::vector<int> &h, const int **dst) -> bool {
             void *q = nullptr;
             if (cudaMalloc(&q, std::max<size_t>(h.size(), 1) * sizeof(int)) != cudaSuccess) return false;
@@ -1024,6 +1124,7 @@ int js_tc_prepare(js_model *mo)
         };
         if (!up(slot_base, &t.lay[l].slot_base) || !up(off, &t.lay[l].sched_off) || !up(flat, &t.lay[l].sched)) return JS_ERR_CUDA;
         t.lay[l].ch = ch;
+        t.lay[l].n_sched = n_sched;
         t.lay[l].slots_per_mt = slots;
         max_slots = std::max(max_slots, slots * MTmax);
         part_floats = std::max(part_floats, (size_t)slots * MTmax * BM * bn);
@@ -1049,12 +1150,9 @@ int js_tc_prepare(js_model *mo)
     t.tmA = (const CUtensorMap *)pa;
     t.tmW = (const CUtensorMap *)pw;
 
-    int meta_ints = 0;
-    for (int l = 0; l <= L; ++l) meta_ints += 3 * t.lay[l].nt;
-    if (meta_ints * 4 > META_MAX_BYTES) return 0;
-    t.smem_bytes = RING_BYTES + STAGING_BYTES + 1024 + ((meta_ints * 4 + 127) & ~127);
+    t.smem_bytes = 1024 + t.ring_bytes + t.aux_bytes + meta_bytes;
     // the attribute belongs to the function, not to a model: always allow the largest request
-    const int smem = RING_BYTES + STAGING_BYTES + 1024 + META_MAX_BYTES;
+    const int smem = SMEM_DYN_MAX;
     if (cudaFuncSetAttribute(made_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
         cudaGetLastError();      // not sticky: the CUDA-core kernels will serve this model
         return 0;
