@@ -323,6 +323,20 @@ struct TcEngine {
                 advance_stage();
             }
         }
+        // The next phase starts with a round trip to HBM for its first weight blocks, while every
+        // CTA waits.  Ask L2 for them now: weights depend on nothing, and this thread is idle until
+        // the grid barrier.  (The same tile range is assumed for the next layer; a wrong guess only
+        // wastes the hint.)
+        {
+            const int ln = (l == m.L) ? 0 : l + 1;
+            const TcLayer &nx = t.lay[ln];
+            int e2, e2_end, lo2 = 0, hi2 = nx.nt;
+            unit_list(ln, MT, e2, e2_end);
+            Unit v;
+            if (next_unit(ln, e2, e2_end, lo2, hi2, MT, v))
+                for (int kb = v.kb0; kb < v.kb1 && kb < v.kb0 + t.n_stages; ++kb)
+                    tma_prefetch_2d(t.tmW + ln, kb * BK, v.nt * nx.bn);
+        }
     }
 
     __device__ void mma_issuer(int l, int nt_lo, int nt_hi, int MT)
@@ -388,25 +402,27 @@ struct TcEngine {
     // owner: bounded wait until this warp's row quadrant of every partial of the tile is stored
     __device__ bool wait_partials(int slot, int nparts)
     {
+        // lane p polls the flag of partial p: one round trip for all of them instead of one each
+        const int q = warp & 3;
         int ok = 1;
-        if (lane == 0) {
-            const int q = warp & 3;
-            for (int p = 0; p < nparts && ok; ++p) {
-                const unsigned *f = t.pflags + (size_t)(slot + p) * 4 + q;
-                uint64_t t0 = 0;
-                for (unsigned i = 0; ld_acquire_u32(f) != stamp; ++i) {
-                    if ((i & 15u) == 15u) {
-                        if (t0 == 0) t0 = global_ns();
-                        if (ld_volatile_i32(&r.ctl->abort) != 0 || global_ns() - t0 > MBAR_WAIT_NS) {
-                            atomicExch(&r.ctl->abort, 1);
-                            ok = 0;
-                            break;
-                        }
+        for (int p0 = 0; p0 < nparts && ok; p0 += 32) {
+            const bool mine = p0 + lane < nparts;
+            const unsigned *f = t.pflags + (size_t)(slot + p0 + (mine ? lane : 0)) * 4 + q;
+            uint64_t t0 = 0;
+            for (unsigned i = 0;; ++i) {
+                const bool set = !mine || ld_acquire_u32(f) == stamp;
+                if (__all_sync(0xffffffffu, set)) break;
+                if ((i & 15u) == 15u) {
+                    if (t0 == 0) t0 = global_ns();
+                    const bool give_up = ld_volatile_i32(&r.ctl->abort) != 0 || global_ns() - t0 > MBAR_WAIT_NS;
+                    if (__any_sync(0xffffffffu, give_up)) {
+                        if (lane == 0) atomicExch(&r.ctl->abort, 1);
+                        ok = 0;
+                        break;
                     }
                 }
             }
         }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
         __threadfence();
         return ok != 0;
     }
@@ -605,13 +621,15 @@ struct TcEngine {
         }
     }
 
+    // NK: the noise kind as a compile-time constant (a per-element branch on it halves the speed
+    // of this loop, which a single warp per scheduler runs)
+    template <int NK>
     __device__ bool epi_binary_tile(const Win &w, int smp, int rw, int n0, int ncols, uint32_t tbase, bool flag,
                                     int parity, bool &wany, int &wfirst)
     {
         const float *bs = sh.bias_s[warp - 2];
         uint8_t *nz = nz_row(), *xs = xs_row();
         const float lut0 = m.lut[0], lut1 = m.lut[1];
-        const int nk = r.nk;
         // columns [clo, chi) of the tile are sampled; the others keep their symbol
         const int clo = max(w.plo - n0, 0), chi = min(min(w.phi, m.T) - n0, ncols);
         if (t.bin_bulk) {
@@ -657,7 +675,7 @@ struct TcEngine {
                         const uint32_t o = (xw >> (8 * k)) & 0xffu;
                         const float z = __uint_as_float(ra[i * 4 + k]) + bb[k];
                         const bool in = (unsigned)(c + k - clo) < (unsigned)(chi - clo);
-                        const uint32_t nv = in ? (uint32_t)js_sample_binary(nk, z, e[k]) : o;
+                        const uint32_t nv = in ? (uint32_t)js_sample_binary(NK, z, e[k]) : o;
                         nw |= nv << (8 * k);
                         enc[k] = nv ? lut1 : lut0;
                     }
@@ -748,7 +766,10 @@ struct TcEngine {
             } else if (kind == EPI_BINARY) {
                 bool wany = false;
                 int wfirst = INT_MAX;
-                if (!epi_binary_tile(w, bsmp, row, n0, bcols, tbase, flag, parity, wany, wfirst)) { dead = true; break; }
+                const bool fine = r.nk == JS_NOISE_LOGISTIC
+                    ? epi_binary_tile<JS_NOISE_LOGISTIC>(w, bsmp, row, n0, bcols, tbase, flag, parity, wany, wfirst)
+                    : epi_binary_tile<JS_NOISE_UNIFORM_ICDF>(w, bsmp, row, n0, bcols, tbase, flag, parity, wany, wfirst);
+                if (!fine) { dead = true; break; }
                 if (wany) { any_changed = true; first = min(first, wfirst); }
             } else {
                 float best = -INFINITY;

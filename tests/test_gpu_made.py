@@ -82,7 +82,7 @@ CAT = si.scaled(si.CONFIGS["made_cat"], D=24, H=(128, 96), batch=9)
 CHAIN = si.scaled(si.CONFIGS["made_4096"], D=256, H=(256, 256, 256, 256), batch=130, w_var_scale=4.0)
 
 # long K ranges with few tiles: the tensor-core kernels cut every tile's K loop into several work units
-SPLIT = si.scaled(si.CONFIGS["made_784"], D=1024, H=(1024, 1024), batch=130, w_var_scale=3.0)
+SPLIT = si.scaled(si.CONFIGS["made_784"], D=512, H=(2688, 2688), batch=130, w_var_scale=3.0)
 
 CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN, "split": SPLIT}
 # kernel path: 1 = CUDA-core kernels, 0 = tensor-core kernels (bf16 models only)
