@@ -160,6 +160,8 @@ int common_scratch(js_model *m, int T)
 {
     int rc;
     if ((rc = dev_alloc<JsCtl>(m, &m->ctl, 1, true)) != JS_OK) return rc;
+    CU_TRY(cudaHostAlloc((void **)&m->h_result, sizeof(JsCtl), cudaHostAllocMapped));
+    CU_TRY(cudaHostGetDevicePointer((void **)&m->d_result, m->h_result, 0));
     if ((rc = dev_alloc<int>(m, &m->smp_changed, 2 * (size_t)m->rows, true)) != JS_OK) return rc;
     if ((rc = dev_alloc<int>(m, &m->smp_state, 2 * (size_t)m->rows, true)) != JS_OK) return rc;
     if ((rc = dev_alloc<int>(m, &m->perm, 2 * (size_t)m->rows, true)) != JS_OK) return rc;
@@ -193,7 +195,12 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
     r.spin_limit = (unsigned)m->opt_spin_limit;
     r.trace = m->opt_trace ? m->trace : nullptr;
     if (r.trace) CU_TRY(cudaMemsetAsync(m->trace, 0, sizeof(unsigned long long) * 2 * JS_TRACE_PHASES * JS_TRACE_SLOTS, st));
-    CU_TRY(cudaMemsetAsync(m->ctl, 0, sizeof(JsCtl), st));
+    // a call that ended normally left the control block zeroed
+    if (!m->ctl_clean) CU_TRY(cudaMemsetAsync(m->ctl, 0, sizeof(JsCtl), st));
+    m->ctl_clean = false;
+    r.result = m->d_result;
+    const int NOT_REPORTED = -1000000;
+    m->h_result->status = NOT_REPORTED;
 
     int used_path = 1;
     int rc_launch;
@@ -225,9 +232,13 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
         snprintf(g_cuda_err, sizeof g_cuda_err, "kernel launch: %s", cudaGetErrorString((cudaError_t)rc_launch));
         return JS_ERR_CUDA;
     }
-    JsCtl h;
-    CU_TRY(cudaMemcpyAsync(&h, m->ctl, sizeof h, cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaStreamSynchronize(st));
+    const JsCtl h = *m->h_result;
+    if (h.status == NOT_REPORTED) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "the kernel ended without reporting");
+        return JS_ERR_CUDA;
+    }
+    m->ctl_clean = h.status >= 0;
     m->stats.iterations = h.iterations;
     m->stats.final_frontier = h.frontier;
     m->stats.tiles_issued = (long long)h.tiles_issued;
@@ -303,6 +314,7 @@ void js_model_destroy(js_model *m)
 {
     if (!m) return;
     for (void *p : m->allocs) cudaFree(p);
+    if (m->h_result) cudaFreeHost(m->h_result);
     delete m;
 }
 

@@ -28,6 +28,7 @@ struct JsCtl {
     int live;               // samples still iterating (tensor-core path)
     int compactions;        // times the working batch was compacted
     unsigned long long tiles_issued, tiles_skipped;
+    unsigned exit_count;    // CTAs that have left; the last one reports and clears the block
 };
 
 // Device view of a masked MLP.  Layer l maps a[l] (width n[l]) to a[l+1].
@@ -66,6 +67,7 @@ struct RunArgs {
     int frontier_skip, seq_skip, compact;
     unsigned spin_limit;
     JsCtl *ctl;
+    JsCtl *result;            // host memory mapped into the device: the last CTA to leave copies ctl here
     unsigned long long *trace;   // [2 CTAs][JS_TRACE_PHASES][JS_TRACE_SLOTS] globaltimer stamps, or NULL
 };
 

@@ -58,6 +58,9 @@ struct js_model {
     std::vector<void *> allocs;   // every device allocation, freed by js_model_destroy
     std::vector<std::vector<int>> host_deg;
     JsCtl *ctl = nullptr;
+    JsCtl *h_result = nullptr;    // pinned host memory, mapped: the kernels report here
+    JsCtl *d_result = nullptr;    // the same memory as the device sees it
+    bool ctl_clean = false;       // the last call left the control block zeroed
     int *smp_changed = nullptr, *smp_state = nullptr, *perm = nullptr;
     uint8_t *x_old = nullptr, *x_tmp = nullptr;
     unsigned long long *trace = nullptr;

@@ -198,16 +198,35 @@ __device__ DriverResult made_driver(E &e, int T_, const RunArgs &r)
     return res;
 }
 
+// Every CTA adds its statistics; the last one to leave copies the control block to the caller's
+// mapped host memory (so that the host needs no device-to-host copy) and zeroes it, ready for
+// the next launch (so that the host needs no memset either, unless a call ended abnormally).
 __device__ __forceinline__ void driver_finish(const RunArgs &r, const DriverResult &res, unsigned long long issued,
                                               unsigned long long skipped)
 {
-    if (threadIdx.x == 0) {
-        atomicAdd(&r.ctl->tiles_issued, issued);
-        atomicAdd(&r.ctl->tiles_skipped, skipped);
-        if (blockIdx.x == 0) {
-            r.ctl->iterations = res.iterations;
-            r.ctl->frontier = res.frontier;
-            r.ctl->status = res.alive ? res.status : JS_ERR_TIMEOUT;
-        }
+    if (threadIdx.x != 0) return;
+    JsCtl *c = r.ctl;
+    atomicAdd(&c->tiles_issued, issued);
+    atomicAdd(&c->tiles_skipped, skipped);
+    if (blockIdx.x == 0) {
+        c->iterations = res.iterations;
+        c->frontier = res.frontier;
     }
+    if (!res.alive) atomicExch(&c->abort, 1);
+    __threadfence();
+    if (atomicAdd(&c->exit_count, 1u) != gridDim.x - 1) return;
+    __threadfence();
+    // word-wise through volatile pointers: the block was written by other CTAs
+    constexpr int NW = sizeof(JsCtl) / 4;
+    unsigned w[NW];
+    volatile unsigned *cw = reinterpret_cast<volatile unsigned *>(c);
+    for (int i = 0; i < NW; ++i) w[i] = cw[i];
+    JsCtl *o = reinterpret_cast<JsCtl *>(w);
+    o->status = o->abort != 0 ? JS_ERR_TIMEOUT : res.status;     // res.status is the same in every CTA
+    if (r.result) {
+        volatile unsigned *rw = reinterpret_cast<volatile unsigned *>(r.result);
+        for (int i = 0; i < NW; ++i) rw[i] = w[i];
+        __threadfence_system();
+    }
+    for (int i = 0; i < NW; ++i) cw[i] = 0u;
 }

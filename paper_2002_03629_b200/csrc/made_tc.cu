@@ -480,26 +480,6 @@ struct TcEngine {
             if (col + i < N) zout[(size_t)row * N + col + i] = v[i] + bias[col + i];
     }
 
-    // one 256-way position per tile: running argmax of logit + Gumbel noise, lowest index wins ties
-    __device__ void epi_cat_chunk(int sample, int d, int c0, const float (&v)[32], float &best, int &bi)
-    {
-        if (sample < 0) return;
-        const float *bias = m.bias[m.L] + (size_t)d * 256 + c0;
-        const float *gg = r.noise + ((size_t)sample * m.T + d) * 256 + c0;
-#pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-            const float4 b4 = __ldg(reinterpret_cast<const float4 *>(bias + i));
-            const float4 g4 = __ldg(reinterpret_cast<const float4 *>(gg + i));
-            const float s0 = (v[i] + b4.x) + g4.x, s1 = (v[i + 1] + b4.y) + g4.y;
-            const float s2 = (v[i + 2] + b4.z) + g4.z, s3 = (v[i + 3] + b4.w) + g4.w;
-            if (s0 > best) { best = s0; bi = c0 + i; }
-            if (s1 > best) { best = s1; bi = c0 + i + 1; }
-            if (s2 > best) { best = s2; bi = c0 + i + 2; }
-            if (s3 > best) { best = s3; bi = c0 + i + 3; }
-        }
-    }
-
-
     // ---- whole-tile epilogues that go through shared memory so that global accesses are
     // coalesced.  Each epilogue warp owns 32 rows of the tile and an 8 KB staging area holding
     // 32 rows x 256 bytes; 16-byte chunk c of row r sits at chunk c ^ (r & 15) (conflict-free both
@@ -722,6 +702,75 @@ struct TcEngine {
         return true;
     }
 
+    // ---- 256-way output layer: one position per tile, thread = one sample row.  Running argmax of
+    // logit + Gumbel noise over eight chunks of 32 classes, lowest index first among equals.  The
+    // row's noise (1 KB) is asked into L2 before the accumulator is waited for, and the noise of
+    // chunk c+1 is loaded before chunk c is reduced, so that one memory latency is exposed per
+    // tile instead of one per chunk.
+    __device__ void cat_prefetch(int sample, int d)
+    {
+        if (sample < 0) return;
+        const float *gg = r.noise + ((size_t)sample * m.T + d) * 256;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) prefetch_l2(gg + i * 32);
+    }
+    __device__ void epi_cat_tile(int sample, int row, int d, uint32_t tbase, const Win &w, bool flag, int parity,
+                                 bool &any_changed, int &first)
+    {
+        const float *bs = sh.bias_s[warp - 2];
+        const float *gg = r.noise + ((size_t)max(sample, 0) * m.T + d) * 256;
+        float best = -INFINITY;
+        int bi = 0;
+        float4 g4[8], gn[8];
+        if (sample >= 0) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) g4[i] = ld_nc_f4_now(gg + i * 4);
+        }
+#pragma unroll 1
+        for (int c0 = 0; c0 < 256; c0 += 32) {
+            uint32_t ra[32];
+            __syncwarp();
+            tmem_ld32_issue(tbase + (uint32_t)c0, ra);
+            if (sample >= 0 && c0 + 32 < 256) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) gn[i] = ld_nc_f4_now(gg + c0 + 32 + i * 4);
+            }
+            tmem_wait_ld();
+            if (c0 == 256 - 32) release_acc();
+            if (cur_parts > 0) add_partials(ra, c0);
+            if (sample >= 0) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const float4 b4 = *reinterpret_cast<const float4 *>(bs + c0 + i * 4);
+                    const float s0 = (__uint_as_float(ra[4 * i]) + b4.x) + g4[i].x;
+                    const float s1 = (__uint_as_float(ra[4 * i + 1]) + b4.y) + g4[i].y;
+                    const float s2 = (__uint_as_float(ra[4 * i + 2]) + b4.z) + g4[i].z;
+                    const float s3 = (__uint_as_float(ra[4 * i + 3]) + b4.w) + g4[i].w;
+                    if (s0 > best) { best = s0; bi = c0 + 4 * i; }
+                    if (s1 > best) { best = s1; bi = c0 + 4 * i + 1; }
+                    if (s2 > best) { best = s2; bi = c0 + 4 * i + 2; }
+                    if (s3 > best) { best = s3; bi = c0 + 4 * i + 3; }
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) g4[i] = gn[i];
+            }
+        }
+        bool ch = false;
+        if (sample >= 0 && d >= w.plo && d < w.phi) {
+            const size_t at = (size_t)sample * m.T + d;
+            if ((int)__ldcg(r.x + at) != bi) {
+                r.x[at] = (uint8_t)bi;
+                ((__nv_bfloat16 *)m.a[0])[(size_t)row * m.T + d] = __float2bfloat16_rn(m.lut[bi]);
+                ch = true;
+            }
+        }
+        if (flag && ch) {
+            raise_flag(parity, sample);
+            any_changed = true;
+            first = min(first, d);
+        }
+    }
+
     __device__ void epilogue(int l, int kind, const Win &w, bool flag, int parity, float *zout, int nt_lo,
                              int nt_hi, int MT)
     {
@@ -735,7 +784,13 @@ struct TcEngine {
         while (!dead && next_unit(l, e, e_end, nt_lo, nt_hi, MT, u)) {
             const int nt = u.nt, mt = u.mt;
             const bool owner = u.nparts >= 0;
-            if (owner && (kind == EPI_HIDDEN || kind == EPI_BINARY)) load_bias_tile(l, nt * ly.bn, ly.bn);
+            if (owner && kind != EPI_LOGITS) load_bias_tile(l, nt * ly.bn, ly.bn);
+            int csmp = -1;
+            if (owner && kind == EPI_CAT) {
+                const int rw = mt * BM + q * 32 + lane;
+                csmp = rw < live ? perm_cur()[rw] : -1;
+                cat_prefetch(csmp, nt);
+            }
             int bsmp = -1, bcols = 0;
             if (owner && kind == EPI_BINARY) {
                 const int rw = mt * BM + q * 32 + lane;
@@ -771,12 +826,9 @@ struct TcEngine {
                     : epi_binary_tile<JS_NOISE_UNIFORM_ICDF>(w, bsmp, row, n0, bcols, tbase, flag, parity, wany, wfirst);
                 if (!fine) { dead = true; break; }
                 if (wany) { any_changed = true; first = min(first, wfirst); }
+            } else if (kind == EPI_CAT) {
+                epi_cat_tile(csmp, row, nt, tbase, w, flag, parity, any_changed, first);
             } else {
-                float best = -INFINITY;
-                int bi = 0;
-                bool ch = false;
-                int fc = INT_MAX;
-                const int sample = (kind == EPI_CAT && row < live) ? perm_cur()[row] : -1;
                 for (int c0 = 0; c0 < ly.bn; c0 += 32) {
                     float v[32];
                     {
@@ -787,22 +839,7 @@ struct TcEngine {
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(ra[i]);
                     }
-                    if (kind == EPI_LOGITS) epi_logits(zout, row, n0, c0, v);
-                    else epi_cat_chunk(sample, nt, c0, v, best, bi);
-                }
-                if (sample >= 0 && nt >= w.plo && nt < w.phi) {
-                    const size_t at = (size_t)sample * m.T + nt;
-                    if ((int)r.x[at] != bi) {
-                        r.x[at] = (uint8_t)bi;
-                        ((__nv_bfloat16 *)m.a[0])[(size_t)row * m.T + nt] = __float2bfloat16_rn(m.lut[bi]);
-                        ch = true;
-                        fc = nt;
-                    }
-                }
-                if (flag && ch) {
-                    raise_flag(parity, sample);
-                    any_changed = true;
-                    first = min(first, fc);
+                    epi_logits(zout, row, n0, c0, v);
                 }
                 release_acc();
             }
