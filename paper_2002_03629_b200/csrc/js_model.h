@@ -29,6 +29,7 @@ struct TcDev {
     TcLayer lay[JS_MAXL + 1];
     int stage_bytes, n_stages, smem_bytes;
     int ring_bytes, aux_bytes;   // shared memory: operand ring, then the epilogues' auxiliary buffer
+    int cat_rows;                // 256-way outputs: the first cat_rows rows of a tile get their noise through shared memory
     int bin_bulk;                // binary output rows are 16-byte granular: moved by bulk copies
     int grid;                    // CTAs the schedules were built for (the launch uses exactly this)
     float *partials;             // [slot][columns/4][128 rows] float4: fp32 partial sums of non-owning chunks

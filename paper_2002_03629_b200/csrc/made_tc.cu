@@ -39,6 +39,7 @@ constexpr int MAX_STAGES = 6;
 // binary output tiles: per sample row 128 noise values and 128 symbols, rows padded by 16 bytes
 constexpr int BIN_NZ_ROW = 512 + 16, BIN_XS_ROW = 128 + 16;
 constexpr int BIN_NZ_BYTES = BM * BIN_NZ_ROW, BIN_XS_BYTES = BM * BIN_XS_ROW;
+constexpr int CAT_ROW = 1024 + 16;     // 256-way output tiles: a sample row's noise, padded
 // Shared memory after the 1 KB alignment slack: operand ring | auxiliary buffer | tile metadata.
 // The auxiliary buffer is the staging area of the hidden-layer epilogues and, in models with
 // binary outputs, also holds the noise and symbol rows of an output tile (never both at once).
@@ -232,8 +233,10 @@ struct TcEngine {
     }
 
     __device__ int kb_end_of(int l, int nt) const { return meta[sh.off[l] + nt]; }
-    __device__ int dmin_of(int l, int nt) const { return meta[sh.off[l] + t.lay[l].nt + nt]; }
-    __device__ int dmax_of(int l, int nt) const { return meta[sh.off[l] + 2 * t.lay[l].nt + nt]; }
+    // a 256-way output tile is one position: its degrees need no table
+    __device__ bool one_pos_tiles(int l) const { return l == m.L && m.C == 256; }
+    __device__ int dmin_of(int l, int nt) const { return one_pos_tiles(l) ? nt + 1 : meta[sh.off[l] + t.lay[l].nt + nt]; }
+    __device__ int dmax_of(int l, int nt) const { return one_pos_tiles(l) ? nt + 1 : meta[sh.off[l] + 2 * t.lay[l].nt + nt]; }
 
     __device__ uint8_t *stage_a(int s) const { return ring + (size_t)s * t.stage_bytes; }
     __device__ uint8_t *stage_b(int s) const { return ring + (size_t)s * t.stage_bytes + A_BYTES; }
@@ -525,7 +528,7 @@ struct TcEngine {
     // and 16-byte chunk (lane & 15) = four consecutive columns.  Their loops are kept rolled: these
     // kernels are instruction-cache bound when every path is unrolled.
 
-    // hidden layer: act(acc + bias) -> bf16, 128 columns in two halves of 64
+    // hidden layer: act(acc + bias) -> bf16, 64 columns at a time
     __device__ void epi_hidden_tile(int l, int mt, int n0, uint32_t tbase)
     {
         uint8_t *stg = my_staging();
@@ -534,10 +537,11 @@ struct TcEngine {
         __nv_bfloat16 *out = (__nv_bfloat16 *)m.a[l + 1];
         const int q = warp & 3, ch = lane & 15, rsel = lane >> 4;
         const int act = m.act;
+        const int halves = t.lay[l].bn / 64;
 #pragma unroll 1
-        for (int half = 0; half < 2; ++half) {
+        for (int half = 0; half < halves; ++half) {
             stage_half(tbase, half);
-            if (half == 1) { release_acc(); if (warp == 2 && lane == 0) trace(6); } else __syncwarp();
+            if (half == halves - 1) { release_acc(); if (warp == 4 && lane == 0) trace(6); } else __syncwarp();
             const int cb = half * 64 + ch * 4;
             const float b0 = bs[cb], b1 = bs[cb + 1], b2 = bs[cb + 2], b3 = bs[cb + 3];
             const int col = n0 + cb;
@@ -546,8 +550,8 @@ struct TcEngine {
                 const int rl = it * 2 + rsel;
                 const float4 v = *reinterpret_cast<const float4 *>(stg + rl * 256 + ((ch ^ (rl & 15)) << 4));
                 const int row = mt * BM + q * 32 + rl;
-                const uint32_t p0 = pack_bf16x2(js_act_fn(act, v.x + b0), js_act_fn(act, v.y + b1));
-                const uint32_t p1 = pack_bf16x2(js_act_fn(act, v.z + b2), js_act_fn(act, v.w + b3));
+                const uint32_t p0 = pack_bf16x2(tc_act_fn(act, v.x + b0), tc_act_fn(act, v.y + b1));
+                const uint32_t p1 = pack_bf16x2(tc_act_fn(act, v.z + b2), tc_act_fn(act, v.w + b3));
                 if (row < live && col < N) *reinterpret_cast<uint2 *>(out + (size_t)row * N + col) = make_uint2(p0, p1);
             }
             __syncwarp();
@@ -618,7 +622,7 @@ struct TcEngine {
         }
         uint32_t diff_any = 0;
         int first = INT_MAX;
-        const bool tr = (warp == 2 && lane == 0);
+        const bool tr = (warp == 4 && lane == 0);
         if (tr) trace(6);
 #pragma unroll 1
         for (int c0 = 0; c0 < BM; c0 += 32) {
@@ -703,10 +707,13 @@ struct TcEngine {
     }
 
     // ---- 256-way output layer: one position per tile, thread = one sample row.  Running argmax of
-    // logit + Gumbel noise over eight chunks of 32 classes, lowest index first among equals.  The
-    // row's noise (1 KB) is asked into L2 before the accumulator is waited for, and the noise of
-    // chunk c+1 is loaded before chunk c is reduced, so that one memory latency is exposed per
-    // tile instead of one per chunk.
+    // logit + Gumbel noise over eight chunks of 32 classes, lowest index first among equals.
+    // This layer is bound by HBM and by its epilogues, and few threads own a valid row when the batch
+    // is small, so plain loads leave little in flight.  Therefore: a row's noise (1 KB) is asked into
+    // L2 one tile ahead, and the rows of the first t.cat_rows rows of the tile (whole warps) come
+    // into shared memory by one bulk copy each, issued before the accumulator is waited for; rows
+    // are padded by 16 bytes so that the row-per-lane reads are conflict-free.  Rows beyond that
+    // load their noise directly, one chunk ahead of the reduction.
     __device__ void cat_prefetch(int sample, int d)
     {
         if (sample < 0) return;
@@ -714,15 +721,34 @@ struct TcEngine {
 #pragma unroll
         for (int i = 0; i < 8; ++i) prefetch_l2(gg + i * 32);
     }
-    __device__ void epi_cat_tile(int sample, int row, int d, uint32_t tbase, const Win &w, bool flag, int parity,
+    __device__ bool cat_in_smem() const { return (warp & 3) * 32 + 32 <= t.cat_rows; }
+    __device__ uint8_t *cat_row() const { return staging + (size_t)((warp & 3) * 32 + lane) * CAT_ROW; }
+    __device__ void cat_fetch_rows(int sample, int d)
+    {
+        if (!cat_in_smem()) return;
+        const int q = warp & 3;
+        __syncwarp();                         // every lane is done with the previous tile's rows
+        const uint32_t tot = __reduce_add_sync(0xffffffffu, sample >= 0 ? 1024u : 0u);
+        if (lane == 0) mbar_expect_tx(&sh.nzbar[q], tot);
+        __syncwarp();
+        if (sample >= 0)
+            bulk_load(smem_u32(cat_row()), r.noise + ((size_t)sample * m.T + d) * 256, 1024u, &sh.nzbar[q]);
+    }
+    __device__ bool epi_cat_tile(int sample, int row, int d, uint32_t tbase, const Win &w, bool flag, int parity,
                                  bool &any_changed, int &first)
     {
         const float *bs = sh.bias_s[warp - 2];
-        const float *gg = r.noise + ((size_t)max(sample, 0) * m.T + d) * 256;
+        const bool smem_rows = cat_in_smem();
+        const float *gg = smem_rows ? reinterpret_cast<const float *>(cat_row())
+                                    : r.noise + ((size_t)max(sample, 0) * m.T + d) * 256;
+        if (smem_rows) {
+            if (!mbar_wait(&sh.nzbar[warp & 3], nzphase, r.ctl)) return false;
+            nzphase ^= 1u;
+        }
         float best = -INFINITY;
         int bi = 0;
         float4 g4[8], gn[8];
-        if (sample >= 0) {
+        if (sample >= 0 && !smem_rows) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) g4[i] = ld_nc_f4_now(gg + i * 4);
         }
@@ -731,9 +757,14 @@ struct TcEngine {
             uint32_t ra[32];
             __syncwarp();
             tmem_ld32_issue(tbase + (uint32_t)c0, ra);
-            if (sample >= 0 && c0 + 32 < 256) {
+            if (sample >= 0) {
+                if (smem_rows) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) gn[i] = ld_nc_f4_now(gg + c0 + 32 + i * 4);
+                    for (int i = 0; i < 8; ++i) g4[i] = *reinterpret_cast<const float4 *>(gg + c0 + i * 4);
+                } else if (c0 + 32 < 256) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) gn[i] = ld_nc_f4_now(gg + c0 + 32 + i * 4);
+                }
             }
             tmem_wait_ld();
             if (c0 == 256 - 32) release_acc();
@@ -751,8 +782,10 @@ struct TcEngine {
                     if (s2 > best) { best = s2; bi = c0 + 4 * i + 2; }
                     if (s3 > best) { best = s3; bi = c0 + 4 * i + 3; }
                 }
+                if (!smem_rows) {
 #pragma unroll
-                for (int i = 0; i < 8; ++i) g4[i] = gn[i];
+                    for (int i = 0; i < 8; ++i) g4[i] = gn[i];
+                }
             }
         }
         bool ch = false;
@@ -769,6 +802,7 @@ struct TcEngine {
             any_changed = true;
             first = min(first, d);
         }
+        return true;
     }
 
     __device__ void epilogue(int l, int kind, const Win &w, bool flag, int parity, float *zout, int nt_lo,
@@ -778,6 +812,7 @@ struct TcEngine {
         const int q = warp & 3;
         bool any_changed = false;
         int first = INT_MAX;
+        bool cat_ahead = false;        // the current tile's noise was asked into L2 during the previous tile
         int e, e_end;
         unit_list(l, MT, e, e_end);
         Unit u;
@@ -789,7 +824,16 @@ struct TcEngine {
             if (owner && kind == EPI_CAT) {
                 const int rw = mt * BM + q * 32 + lane;
                 csmp = rw < live ? perm_cur()[rw] : -1;
-                cat_prefetch(csmp, nt);
+                if (!cat_ahead) cat_prefetch(csmp, nt);          // first tile of the phase
+                cat_fetch_rows(csmp, nt);
+                // the next tile's noise towards L2 while this tile is reduced
+                Unit nx;
+                int e2 = e;
+                cat_ahead = next_unit(l, e2, e_end, nt_lo, nt_hi, MT, nx) && nx.nparts >= 0;
+                if (cat_ahead) {
+                    const int rn = nx.mt * BM + q * 32 + lane;
+                    cat_prefetch(rn < live ? perm_cur()[rn] : -1, nx.nt);
+                }
             }
             int bsmp = -1, bcols = 0;
             if (owner && kind == EPI_BINARY) {
@@ -807,7 +851,7 @@ struct TcEngine {
             }
             if (!mbar_wait(&sh.tfull[acc], aphase, r.ctl)) { dead = true; break; }
             tc_fence_after();
-            if (warp == 2 && lane == 0) trace(3);
+            if (warp == 4 && lane == 0) trace(3);
             const int row = mt * BM + q * 32 + lane;
             const int n0 = nt * ly.bn;
             const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS);
@@ -827,7 +871,7 @@ struct TcEngine {
                 if (!fine) { dead = true; break; }
                 if (wany) { any_changed = true; first = min(first, wfirst); }
             } else if (kind == EPI_CAT) {
-                epi_cat_tile(csmp, row, nt, tbase, w, flag, parity, any_changed, first);
+                if (!epi_cat_tile(csmp, row, nt, tbase, w, flag, parity, any_changed, first)) { dead = true; break; }
             } else {
                 for (int c0 = 0; c0 < ly.bn; c0 += 32) {
                     float v[32];
@@ -846,7 +890,7 @@ struct TcEngine {
             advance_acc();
         }
         bulk_wait_all();          // bulk stores of this phase are complete before the grid barrier
-        if (warp == 2 && lane == 0) trace(4);
+        if (warp == 4 && lane == 0) trace(4);
         if (flag) {
             const bool wany = __any_sync(0xffffffffu, any_changed);
             if (wany) {
@@ -921,12 +965,15 @@ made_tc_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ TcDev 
         for (int l = 0; l <= m.L; ++l) {
             const int nt = t.lay[l].nt;
             if (threadIdx.x == 0) sh.off[l] = off;
+            const bool one_pos = (l == m.L && m.C == 256);
             for (int i = threadIdx.x; i < nt; i += blockDim.x) {
                 meta[off + i] = t.lay[l].kb_end[i];
-                meta[off + nt + i] = t.lay[l].dmin[i];
-                meta[off + 2 * nt + i] = t.lay[l].dmax[i];
+                if (!one_pos) {
+                    meta[off + nt + i] = t.lay[l].dmin[i];
+                    meta[off + 2 * nt + i] = t.lay[l].dmax[i];
+                }
             }
-            off += 3 * nt;
+            off += one_pos ? nt : 3 * nt;
         }
     }
     tc_fence_before();
@@ -1004,10 +1051,32 @@ int js_tc_prepare(js_model *mo)
     const int L = v.L;
     bool wide = (v.C == 256);
     t.stage_bytes = A_BYTES + (wide ? 256 : 128) * BK * 2;
+    // Output-tile width per layer: 256 for 256-way outputs (one position per tile), else 128; hidden
+    // layers with so few 128-wide tiles that three quarters of the SMs would idle use 64 (shorter K
+    // blocks, half the epilogue per CTA, twice the CTAs).
+    int sms_now = 0;
+    {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms_now, cudaDevAttrMultiProcessorCount, dev);
+    }
+    std::vector<int> bns(L + 1);
+    for (int l = 0; l <= L; ++l) {
+        bns[l] = (l == L && wide) ? 256 : 128;
+        if (l < L && (long long)((v.n[l + 1] + 127) / 128) * (mo->rows / BM) * 4 <= sms_now) bns[l] = 64;
+    }
     int meta_ints = 0;
-    for (int l = 0; l <= L; ++l) meta_ints += 3 * ((v.n[l + 1] + ((l == L && wide) ? 256 : 128) - 1) / ((l == L && wide) ? 256 : 128));
+    for (int l = 0; l <= L; ++l)
+        meta_ints += (l == L && wide) ? (v.n[l + 1] + 255) / 256 : 3 * ((v.n[l + 1] + bns[l] - 1) / bns[l]);
     const int meta_bytes = (meta_ints * 4 + 127) & ~127;
-    t.aux_bytes = wide ? STAGING_BYTES : std::max(STAGING_BYTES, BIN_NZ_BYTES + BIN_XS_BYTES);
+    t.aux_bytes = std::max(STAGING_BYTES, BIN_NZ_BYTES + BIN_XS_BYTES);
+    t.cat_rows = 0;
+    if (wide) {
+        // three operand stages; the rest holds as many whole warps of noise rows as fit
+        const int left = SMEM_DYN_MAX - 1024 - 3 * t.stage_bytes - meta_bytes;
+        t.cat_rows = std::min(BM, std::max(0, left / (32 * CAT_ROW)) * 32);
+        t.aux_bytes = std::max(STAGING_BYTES, t.cat_rows * CAT_ROW);
+    }
     t.bin_bulk = (!wide && v.T % 16 == 0) ? 1 : 0;
     t.n_stages = (SMEM_DYN_MAX - 1024 - t.aux_bytes - meta_bytes) / t.stage_bytes;
     if (t.n_stages > (wide ? 3 : 4)) t.n_stages = wide ? 3 : 4;
@@ -1016,7 +1085,7 @@ int js_tc_prepare(js_model *mo)
     std::vector<CUtensorMap> mapsA(L + 1), mapsW(L + 1);
     std::vector<std::vector<int>> kb_all(L + 1);
     for (int l = 0; l <= L; ++l) {
-        const int bn = (l == L && wide) ? 256 : 128;
+        const int bn = bns[l];
         const int N = v.n[l + 1], K = v.n[l], nt = (N + bn - 1) / bn;
         std::vector<int> kb(nt), dmin(nt), dmax(nt);
         const std::vector<int> &dout = mo->host_deg[l + 1], &din = mo->host_deg[l];
@@ -1110,7 +1179,7 @@ int js_tc_prepare(js_model *mo)
             // tile's partial sums have been stored.  Units are taken longest first and put where
             // the CTA finishes earliest.  Inside a CTA: partial chunks first (owners elsewhere
             // wait for them), then owners that wait for nobody, then owners that add partial sums.
-            const int FILL = 6, EPI_PART = 5, EPI_OWN = (l == L ? (bn == 256 ? 24 : 9) : 4), EPI_ADD = 8;
+            const int FILL = 6, EPI_PART = 5, EPI_OWN = (l == L ? (bn == 256 ? 5 : 9) : 4), EPI_ADD = 8;
             struct Item { int code, size, epi, ready; };
             std::vector<std::vector<Item>> lp(G), lo0(G), lo1(G);
             auto finish = [&](int c, const Item *extra, int where) {

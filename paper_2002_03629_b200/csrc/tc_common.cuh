@@ -220,6 +220,16 @@ __device__ __forceinline__ uint32_t instr_desc_bf16(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
+// Activation of the bf16 epilogues.  GELU in its tanh form is  v * sigmoid(2 y),
+// y = sqrt(2/pi) (v + 0.044715 v^3); one exponential and one division of the fast kind:
+// the result is rounded to bf16, which hides their last bits.
+__device__ __forceinline__ float tc_act_fn(int act, float v)
+{
+    if (act == JS_ACT_RELU) return fmaxf(v, 0.0f);
+    const float y2 = 1.5957691216057308f * (v + 0.044715f * v * v * v);
+    return __fdividef(v, 1.0f + __expf(-y2));
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
