@@ -84,7 +84,10 @@ CHAIN = si.scaled(si.CONFIGS["made_4096"], D=256, H=(256, 256, 256, 256), batch=
 # long K ranges with few tiles: the tensor-core kernels cut every tile's K loop into several work units
 SPLIT = si.scaled(si.CONFIGS["made_784"], D=512, H=(2688, 2688), batch=130, w_var_scale=3.0)
 
-CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN, "split": SPLIT}
+# more rows than the 256-way epilogue keeps in shared memory: rows beyond load their noise directly
+CAT_ROWS = si.scaled(si.CONFIGS["made_cat"], D=16, H=(64, 64), batch=100)
+
+CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN, "split": SPLIT, "cat_rows": CAT_ROWS}
 # kernel path: 1 = CUDA-core kernels, 0 = tensor-core kernels (bf16 models only)
 COMBOS = [(n, 1) for n in CASES] + [(n, 0) for n in CASES if n != "tiny"]
 COMBO_IDS = [f"{n}-{'tc' if p == 0 else 'cc'}" for n, p in COMBOS]
