@@ -1224,6 +1224,22 @@ int js_tc_prepare(js_model *mo)
                                  np > 0 ? (int)ready[(size_t)u.mt * nt + u.nt] + 3 : 0};
                 place(it, np > 0 ? 2 : 1);
             }
+            // Where a CTA has several whole tiles whose epilogue lasts longer than a short K loop (the
+            // 256-way argmax), a run of short tiles at the end of its list leaves their epilogues in
+            // the open.  Order such lists short, long, short, long ...: every short tile's epilogue
+            // hides behind the long K loop that follows, and only the last tile's shows.
+            if (ch == (1 << 20) && bn == 256)
+                for (int c = 0; c < G; ++c) {
+                    std::vector<Item> &v0 = lo0[c];
+                    std::stable_sort(v0.begin(), v0.end(), [](const Item &a, const Item &b) { return a.size < b.size; });
+                    std::vector<Item> mix;
+                    for (size_t i = 0, j = v0.size(); i < j;) {
+                        mix.push_back(v0[i++]);
+                        if (i < j) mix.push_back(v0[--j]);
+                    }
+                    // short, longest, next short, next longest ...; the middle of the sorted list comes last
+                    v0 = mix;
+                }
             std::vector<long long> load(G, 0);
             for (int c = 0; c < G; ++c) {
                 load[c] = finish(c, nullptr, 0);
