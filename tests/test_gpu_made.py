@@ -87,7 +87,11 @@ SPLIT = si.scaled(si.CONFIGS["made_784"], D=512, H=(2688, 2688), batch=130, w_va
 # more rows than the 256-way epilogue keeps in shared memory: rows beyond load their noise directly
 CAT_ROWS = si.scaled(si.CONFIGS["made_cat"], D=16, H=(64, 64), batch=100)
 
-CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN, "split": SPLIT, "cat_rows": CAT_ROWS}
+# uniform noise with the inverse-CDF rule on a bf16 model (the tensor-core epilogue has one instance per noise kind)
+BIN_ICDF = si.scaled(si.CONFIGS["made_784"], D=144, H=(128,), batch=40, noise_kind=si.NOISE_UNIFORM_ICDF)
+
+CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN, "split": SPLIT, "cat_rows": CAT_ROWS,
+         "bin_icdf": BIN_ICDF}
 # kernel path: 1 = CUDA-core kernels, 0 = tensor-core kernels (bf16 models only)
 COMBOS = [(n, 1) for n in CASES] + [(n, 0) for n in CASES if n != "tiny"]
 COMBO_IDS = [f"{n}-{'tc' if p == 0 else 'cc'}" for n, p in COMBOS]
