@@ -294,17 +294,18 @@ def run_ours(args, cfg):
             step()
     clocks = sampler.stop() if sampler else None
 
-    # ---- end to end: pinned host noise in, samples out, inside the timed region
+    # ---- end to end: the host-buffer call of the C ABI, pinned host noise in, host samples out; the
+    # upload, the solve and the download are all inside the call and inside the timed region
+    pkg.jacobi_sample_host(model, h_noise, nk, None, mode, block, 0, h_out)       # allocates the staging buffers
+    if not torch.equal(h_out, out.cpu()):
+        raise RuntimeError("jacobi_sample_host and jacobi_sample disagree")
     barrier()
     t_e2e = []
     for _ in range(1 if args.profile else args.steps):
         flush.zero_()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        d_noise.copy_(h_noise, non_blocking=True)
-        step()
-        h_out.copy_(out, non_blocking=True)
-        torch.cuda.synchronize()
+        pkg.jacobi_sample_host(model, h_noise, nk, None, mode, block, 0, h_out)
         t_e2e.append(time.perf_counter() - t0)
     e2e_s = float(sum(t_e2e)) * (args.steps / len(t_e2e))
 

@@ -119,6 +119,24 @@ int jacobi_sample(const js_model *m, int batch, const float *noise_dev, int nk,
                   const uint8_t *init_dev, int mode, int block, int max_iters,
                   uint8_t *out_samples_dev, int32_t *out_iters_dev, void *cuda_stream);
 
+/*
+ * The same solve (Algorithms 1-3) for callers whose noise and samples live in HOST memory.
+ *   noise_host        fp32, same layout as noise_dev above; pinned memory makes the upload
+ *                     asynchronous, pageable memory works too
+ *   init_host         uint8 [batch][T] or NULL (zeros)
+ *   out_samples_host  uint8 [batch][T]; out_iters_host int32 [batch] or NULL
+ * The library owns the device-side staging buffers (allocated on the first call of a model,
+ * sized for its max_batch) and a copy stream.  The upload of the noise runs beside the first
+ * hidden layers: noise is not needed before the first sampling step (Appendix A.3: it only
+ * turns the conditional of a position into a symbol), and the tensor-core kernel waits
+ * (bounded) for it there; the other kernels start after the upload.  The call returns when
+ * the samples are in out_samples_host.  Return codes as jacobi_sample; the caller's buffers
+ * are only read (noise, init) or written (samples, iters) during the call.
+ */
+int jacobi_sample_host(const js_model *m, int batch, const float *noise_host, int nk,
+                       const uint8_t *init_host, int mode, int block, int max_iters,
+                       uint8_t *out_samples_host, int32_t *out_iters_host, void *cuda_stream);
+
 /* Strict feedforward order (Eq. 1): T steps, each a forward pass of the same kernels of
  * which one position is kept. */
 int sequential_sample(const js_model *m, int batch, const float *noise_dev, int nk,

@@ -11,6 +11,6 @@ from .binding import (  # noqa: F401
     JS_ACT_RELU, JS_ACT_GELU_TANH, JS_F32, JS_BF16,
     JS_OK, JS_NOT_CONVERGED, JS_ERR_ARG, JS_ERR_UNSUPPORTED, JS_ERR_CUDA, JS_ERR_TIMEOUT,
     JS_OPT_FRONTIER_SKIP, JS_OPT_SEQ_SKIP, JS_OPT_SPIN_LIMIT, JS_OPT_PATH, JS_OPT_COMPACT, JS_OPT_TRACE,
-    JsError, Model, load_library, jacobi_sample, sequential_sample, js_forward_logits,
+    JsError, Model, load_library, jacobi_sample, jacobi_sample_host, sequential_sample, js_forward_logits,
     jacobi_sample_noalloc, noalloc_scratch_needed, noalloc_scratch_limit,
 )

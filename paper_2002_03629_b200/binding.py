@@ -68,6 +68,7 @@ def load_library():
     lib.js_model_destroy.argtypes = [vp]
     lib.js_model_destroy.restype = None
     lib.jacobi_sample.argtypes = [vp, ip, vp, ip, vp, ip, ip, ip, vp, vp, vp]
+    lib.jacobi_sample_host.argtypes = [vp, ip, vp, ip, vp, ip, ip, ip, vp, vp, vp]
     lib.sequential_sample.argtypes = [vp, ip, vp, ip, vp, vp]
     lib.js_forward_logits.argtypes = [vp, ip, vp, vp, vp]
     lib.js_set_option.argtypes = [vp, ip, ip]
@@ -210,6 +211,26 @@ def jacobi_sample(model: Model, noise: torch.Tensor, nk: int, init: Optional[tor
         max_iters, _dev(out_samples, torch.uint8, "out_samples"), _dev(out_iters, torch.int32, "out_iters"),
         _stream_ptr(stream))
     return _check(rc, "jacobi_sample")
+
+
+def _host(t: Optional[torch.Tensor], dtype, what: str):
+    if t is None:
+        return None
+    if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise JsError(JS_ERR_ARG, f"{what}: expected a contiguous CPU tensor of {dtype}")
+    return C.c_void_p(t.data_ptr())
+
+
+def jacobi_sample_host(model: Model, noise: torch.Tensor, nk: int, init: Optional[torch.Tensor], mode: int,
+                       block: int, max_iters: int, out_samples: torch.Tensor,
+                       out_iters: Optional[torch.Tensor] = None, stream=None) -> int:
+    """jacobi_sample_host of the C ABI: CPU tensors in and out (pinned ones upload asynchronously)."""
+    batch = out_samples.shape[0]
+    rc = load_library().jacobi_sample_host(
+        model._h, batch, _host(noise, torch.float32, "noise"), nk, _host(init, torch.uint8, "init"), mode, block,
+        max_iters, _host(out_samples, torch.uint8, "out_samples"), _host(out_iters, torch.int32, "out_iters"),
+        _stream_ptr(stream))
+    return _check(rc, "jacobi_sample_host")
 
 
 def sequential_sample(model: Model, noise: torch.Tensor, nk: int, out_samples: torch.Tensor, stream=None) -> int:

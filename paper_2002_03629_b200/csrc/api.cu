@@ -315,6 +315,10 @@ void js_model_destroy(js_model *m)
     if (!m) return;
     for (void *p : m->allocs) cudaFree(p);
     if (m->h_result) cudaFreeHost(m->h_result);
+    if (m->h_nflag) cudaFreeHost(m->h_nflag);
+    if (m->ev_main) cudaEventDestroy(m->ev_main);
+    if (m->ev_copy) cudaEventDestroy(m->ev_copy);
+    if (m->copy_stream) cudaStreamDestroy(m->copy_stream);
     delete m;
 }
 
@@ -336,6 +340,78 @@ int jacobi_sample(const js_model *cm, int batch, const float *noise_dev, int nk,
     r.block = block; r.max_iters = max_iters;
     r.x = out_samples_dev; r.out_iters = out_iters_dev;
     int rc = run_made(m, r, (cudaStream_t)cuda_stream);
+    return rc;
+}
+
+// device staging, copy stream and events of the host-buffer entry point, on first use
+static int ensure_host_staging(js_model *m)
+{
+    if (m->copy_stream) return JS_OK;
+    const int T = m->kind == 0 ? m->made.T : m->conv_T;
+    const int C = m->kind == 0 ? m->made.C : m->conv_C;
+    int rc;
+    if ((rc = dev_alloc<float>(m, &m->st_noise, (size_t)m->max_batch * T * C, false)) != JS_OK) return rc;
+    if ((rc = dev_alloc<uint8_t>(m, &m->st_x, (size_t)m->max_batch * T, false)) != JS_OK) return rc;
+    if ((rc = dev_alloc<uint8_t>(m, &m->st_init, (size_t)m->max_batch * T, false)) != JS_OK) return rc;
+    if ((rc = dev_alloc<int32_t>(m, &m->st_iters, (size_t)m->max_batch, false)) != JS_OK) return rc;
+    if ((rc = dev_alloc<unsigned>(m, &m->d_nflag, 4, true)) != JS_OK) return rc;
+    CU_TRY(cudaHostAlloc((void **)&m->h_nflag, sizeof(unsigned), cudaHostAllocDefault));
+    CU_TRY(cudaEventCreateWithFlags(&m->ev_main, cudaEventDisableTiming));
+    CU_TRY(cudaEventCreateWithFlags(&m->ev_copy, cudaEventDisableTiming));
+    CU_TRY(cudaStreamCreateWithFlags(&m->copy_stream, cudaStreamNonBlocking));
+    return JS_OK;
+}
+
+int jacobi_sample_host(const js_model *cm, int batch, const float *noise_host, int nk, const uint8_t *init_host,
+                       int mode, int block, int max_iters, uint8_t *out_samples_host, int32_t *out_iters_host,
+                       void *cuda_stream)
+{
+    js_model *m = const_cast<js_model *>(cm);
+    if (!m || !noise_host || !out_samples_host) return JS_ERR_ARG;
+    if (batch < 1 || batch > m->max_batch) return JS_ERR_ARG;
+    if (mode < JS_JACOBI || mode > JS_JACOBI_GS) return JS_ERR_ARG;
+    if (!noise_kind_ok(m, nk)) return JS_ERR_ARG;
+    const int T = m->kind == 0 ? m->made.T : m->conv_T;
+    const int C = m->kind == 0 ? m->made.C : m->conv_C;
+    if ((mode == JS_GS_JACOBI || mode == JS_JACOBI_GS) && (block < 1 || block > T)) return JS_ERR_ARG;
+    int rc = ensure_host_staging(m);
+    if (rc != JS_OK) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream, cs = m->copy_stream;
+    // the uploads start once the work the caller queued on `st` before this call is done
+    CU_TRY(cudaEventRecord(m->ev_main, st));
+    CU_TRY(cudaStreamWaitEvent(cs, m->ev_main, 0));
+    if (init_host) {
+        CU_TRY(cudaMemcpyAsync(m->st_init, init_host, (size_t)batch * T, cudaMemcpyHostToDevice, cs));
+        CU_TRY(cudaEventRecord(m->ev_copy, cs));
+        CU_TRY(cudaStreamWaitEvent(st, m->ev_copy, 0));       // the start iterate is needed at once
+    }
+    CU_TRY(cudaMemcpyAsync(m->st_noise, noise_host, (size_t)batch * T * C * sizeof(float), cudaMemcpyHostToDevice, cs));
+    // copies of one stream run in order: this word changes after the noise has arrived
+    *m->h_nflag = ++m->n_uploads;
+    CU_TRY(cudaMemcpyAsync(m->d_nflag, m->h_nflag, sizeof(unsigned), cudaMemcpyHostToDevice, cs));
+    RunArgs r;
+    memset(&r, 0, sizeof r);
+    r.batch = batch; r.noise = m->st_noise; r.nk = nk; r.init = init_host ? m->st_init : nullptr;
+    r.kmode = mode == JS_JACOBI ? KM_JACOBI : mode == JS_GAUSS_SEIDEL ? KM_SEQ : mode == JS_GS_JACOBI ? KM_GS_JACOBI
+                                                                                                        : KM_JACOBI_GS;
+    r.block = block; r.max_iters = max_iters;
+    r.x = m->st_x; r.out_iters = m->st_iters;
+    // only the tensor-core kernel of the masked MLPs waits for the noise by itself
+    const bool overlap = m->kind == 0 && m->tc_ok && m->opt_path == 0 && r.kmode != KM_JACOBI_GS;
+    if (overlap) {
+        r.noise_ready = m->d_nflag;
+        r.noise_stamp = m->n_uploads;
+    } else {
+        CU_TRY(cudaEventRecord(m->ev_copy, cs));
+        CU_TRY(cudaStreamWaitEvent(st, m->ev_copy, 0));
+    }
+    rc = run_made(m, r, st);
+    CU_TRY(cudaStreamSynchronize(cs));
+    if (rc < 0) return rc;
+    CU_TRY(cudaMemcpyAsync(out_samples_host, m->st_x, (size_t)batch * T, cudaMemcpyDeviceToHost, st));
+    if (out_iters_host)
+        CU_TRY(cudaMemcpyAsync(out_iters_host, m->st_iters, (size_t)batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
     return rc;
 }
 

@@ -67,6 +67,8 @@ struct RunArgs {
     int frontier_skip, seq_skip, compact;
     unsigned spin_limit;
     JsCtl *ctl;
+    const unsigned *noise_ready;   // NULL, or a word that takes the value noise_stamp once `noise` has arrived
+    unsigned noise_stamp;
     JsCtl *result;            // host memory mapped into the device: the last CTA to leave copies ctl here
     unsigned long long *trace;   // [2 CTAs][JS_TRACE_PHASES][JS_TRACE_SLOTS] globaltimer stamps, or NULL
 };

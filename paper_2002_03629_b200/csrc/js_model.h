@@ -62,6 +62,14 @@ struct js_model {
     JsCtl *h_result = nullptr;    // pinned host memory, mapped: the kernels report here
     JsCtl *d_result = nullptr;    // the same memory as the device sees it
     bool ctl_clean = false;       // the last call left the control block zeroed
+    // host-buffer entry point: device staging, copy stream, "noise has arrived" word
+    float *st_noise = nullptr;
+    uint8_t *st_x = nullptr, *st_init = nullptr;
+    int32_t *st_iters = nullptr;
+    unsigned *d_nflag = nullptr, *h_nflag = nullptr;
+    unsigned n_uploads = 0;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_main = nullptr, ev_copy = nullptr;
     int *smp_changed = nullptr, *smp_state = nullptr, *perm = nullptr;
     uint8_t *x_old = nullptr, *x_tmp = nullptr;
     unsigned long long *trace = nullptr;

@@ -76,6 +76,7 @@ struct TcEngine {
     int acc = 0;
     uint32_t aphase = 0;
     uint32_t nzphase = 0;
+    bool noise_here = false;       // the uploaded noise has been seen to be complete
     bool dead = false;
     uint32_t tmem_base = 0;
     // working batch: rows [0, live) of the activation buffers hold samples perm[pcur][row]
@@ -810,6 +811,31 @@ struct TcEngine {
     {
         const TcLayer &ly = t.lay[l];
         const int q = warp & 3;
+        // noise that is still on its way from the host (jacobi_sample_host): the first sampling
+        // epilogue waits for it, bounded
+        if (r.noise_ready != nullptr && !noise_here && (kind == EPI_BINARY || kind == EPI_CAT)) {
+            int ok = 1;
+            if (lane == 0) {
+                uint64_t t0 = 0;
+                for (unsigned i = 0;; ++i) {
+                    unsigned v;
+                    asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(r.noise_ready) : "memory");
+                    if (v == r.noise_stamp) break;
+                    if ((i & 15u) == 15u) {
+                        if (t0 == 0) t0 = global_ns();
+                        if (ld_volatile_i32(&r.ctl->abort) != 0 || global_ns() - t0 > MBAR_WAIT_NS) {
+                            atomicExch(&r.ctl->abort, 1);
+                            ok = 0;
+                            break;
+                        }
+                    }
+                    __nanosleep(200);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) dead = true;
+            noise_here = true;
+        }
         bool any_changed = false;
         int first = INT_MAX;
         bool cat_ahead = false;        // the current tile's noise was asked into L2 during the previous tile
