@@ -14,6 +14,7 @@ struct TcLayer {
     const int *dmax;
     int bn;
     int nt;
+    int stage_bytes, n_stages;   // this layer's cut of the operand ring
     // split-K: the K blocks of tile nt are cut into chunks of `ch` blocks, each chunk a work unit
     // of its own; the last chunk owns the tile and adds the others' fp32 partial sums in order
     int ch;

@@ -72,7 +72,8 @@ struct TcEngine {
     int warp, lane;
     // pipeline state, advanced identically by the roles that share it
     int stage = 0;
-    uint32_t sphase = 0;
+    uint32_t spar = 0;             // bit s: parity of the next use of ring stage s
+    int cur_stages = 1, cur_stage_bytes = 0;      // ring geometry of the current layer
     int acc = 0;
     uint32_t aphase = 0;
     uint32_t nzphase = 0;
@@ -239,11 +240,23 @@ struct TcEngine {
     __device__ int dmin_of(int l, int nt) const { return one_pos_tiles(l) ? nt + 1 : meta[sh.off[l] + t.lay[l].nt + nt]; }
     __device__ int dmax_of(int l, int nt) const { return one_pos_tiles(l) ? nt + 1 : meta[sh.off[l] + 2 * t.lay[l].nt + nt]; }
 
-    __device__ uint8_t *stage_a(int s) const { return ring + (size_t)s * t.stage_bytes; }
-    __device__ uint8_t *stage_b(int s) const { return ring + (size_t)s * t.stage_bytes + A_BYTES; }
+    // The ring is cut anew for every layer: narrower weight tiles give more, smaller stages in the
+    // same memory.  That is safe because the ring is drained at every phase boundary, and because
+    // the parity of a stage's barriers is kept per stage (the u-th use of stage s waits for
+    // completion u of full[s] and for completion u-1 of empty[s], whatever the order of use).
+    __device__ void ring_for_layer(int l)
+    {
+        cur_stages = t.lay[l].n_stages;
+        cur_stage_bytes = t.lay[l].stage_bytes;
+        stage = 0;
+    }
+    __device__ uint8_t *stage_a(int s) const { return ring + (size_t)s * cur_stage_bytes; }
+    __device__ uint8_t *stage_b(int s) const { return ring + (size_t)s * cur_stage_bytes + A_BYTES; }
+    __device__ uint32_t stage_parity() const { return (spar >> stage) & 1u; }
     __device__ void advance_stage()
     {
-        if (++stage == t.n_stages) { stage = 0; sphase ^= 1u; }
+        spar ^= 1u << stage;
+        if (++stage == cur_stages) stage = 0;
     }
     __device__ void advance_acc()
     {
@@ -313,6 +326,7 @@ struct TcEngine {
         const TcLayer &ly = t.lay[l];
         const CUtensorMap *ma = t.tmA + l, *mw = t.tmW + l;
         const uint32_t bytes = A_BYTES + ly.bn * BK * 2;
+        ring_for_layer(l);
         trace(0);
         int e, e_end;
         unit_list(l, MT, e, e_end);
@@ -320,7 +334,7 @@ struct TcEngine {
         while (!dead && next_unit(l, e, e_end, nt_lo, nt_hi, MT, u)) {
             issued++;
             for (int kb = u.kb0; kb < u.kb1; ++kb) {
-                if (!mbar_wait(&sh.empty[stage], sphase ^ 1u, r.ctl)) { dead = true; break; }
+                if (!mbar_wait(&sh.empty[stage], stage_parity() ^ 1u, r.ctl)) { dead = true; break; }
                 mbar_expect_tx(&sh.full[stage], bytes);
                 tma_load_2d(smem_u32(stage_a(stage)), ma, &sh.full[stage], kb * BK, u.mt * BM);
                 tma_load_2d(smem_u32(stage_b(stage)), mw, &sh.full[stage], kb * BK, u.nt * ly.bn);
@@ -338,7 +352,7 @@ struct TcEngine {
             unit_list(ln, MT, e2, e2_end);
             Unit v;
             if (next_unit(ln, e2, e2_end, lo2, hi2, MT, v))
-                for (int kb = v.kb0; kb < v.kb1 && kb < v.kb0 + t.n_stages; ++kb)
+                for (int kb = v.kb0; kb < v.kb1 && kb < v.kb0 + nx.n_stages; ++kb)
                     tma_prefetch_2d(t.tmW + ln, kb * BK, v.nt * nx.bn);
         }
     }
@@ -347,6 +361,7 @@ struct TcEngine {
     {
         const TcLayer &ly = t.lay[l];
         const uint32_t idesc = instr_desc_bf16(ly.bn);
+        ring_for_layer(l);
         int e, e_end;
         unit_list(l, MT, e, e_end);
         Unit u;
@@ -356,7 +371,7 @@ struct TcEngine {
             tc_fence_after();
             const uint32_t d_tmem = tmem_base + (uint32_t)(acc * ACC_COLS);
             for (int kb = u.kb0; kb < u.kb1; ++kb) {
-                if (!mbar_wait(&sh.full[stage], sphase, r.ctl)) { dead = true; break; }
+                if (!mbar_wait(&sh.full[stage], stage_parity(), r.ctl)) { dead = true; break; }
                 tc_fence_after();
                 if (first) { trace(1); first = false; }
                 const uint64_t adesc = smem_desc_sw128(smem_u32(stage_a(stage)));
@@ -1135,6 +1150,8 @@ int js_tc_prepare(js_model *mo)
         }
         t.lay[l].bn = bn;
         t.lay[l].nt = nt;
+        t.lay[l].stage_bytes = A_BYTES + bn * BK * 2;
+        t.lay[l].n_stages = std::min(MAX_STAGES, t.ring_bytes / t.lay[l].stage_bytes);
         kb_all[l] = kb;
         if (!encode_map(&mapsA[l], v.a[l], mo->rows, K, BM)) return 0;
         if (!encode_map(&mapsW[l], v.W[l], N, K, bn)) return 0;
