@@ -503,7 +503,8 @@ struct TcEngine {
     // coalesced.  Each epilogue warp owns 32 rows of the tile and an 8 KB staging area holding
     // 32 rows x 256 bytes; 16-byte chunk c of row r sits at chunk c ^ (r & 15) (conflict-free both
     // for the row-per-lane writes and for the row-wise reads).
-    __device__ uint8_t *my_staging() const { return staging + (size_t)(warp - 2) * 8192; }
+    // (at the end of the auxiliary buffer: the part before it serves hidden layers as extra ring stages)
+    __device__ uint8_t *my_staging() const { return staging + (t.aux_bytes - STAGING_BYTES) + (size_t)(warp - 2) * 8192; }
 
     __device__ void load_bias_tile(int l, int n0, int bn)
     {
@@ -1151,7 +1152,11 @@ int js_tc_prepare(js_model *mo)
         t.lay[l].bn = bn;
         t.lay[l].nt = nt;
         t.lay[l].stage_bytes = A_BYTES + bn * BK * 2;
-        t.lay[l].n_stages = std::min(MAX_STAGES, t.ring_bytes / t.lay[l].stage_bytes);
+        // hidden layers need only the staging area at the end of the auxiliary buffer: the ring may
+        // run into the rest of it (an SM keeps about three stages in flight, and 96 KB in flight are
+        // not quite enough to saturate its 108 GB/s)
+        const int ring_cap = t.ring_bytes + (l < L ? t.aux_bytes - STAGING_BYTES : 0);
+        t.lay[l].n_stages = std::min(MAX_STAGES, ring_cap / t.lay[l].stage_bytes);
         kb_all[l] = kb;
         if (!encode_map(&mapsA[l], v.a[l], mo->rows, K, BM)) return 0;
         if (!encode_map(&mapsW[l], v.W[l], N, K, bn)) return 0;
