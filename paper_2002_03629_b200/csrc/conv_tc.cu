@@ -69,11 +69,24 @@ struct ConvEngine {
         lane = threadIdx.x & 31;
     }
 
+    // optional device timeline (JS_OPT_TRACE, js_get_trace): first and last CTA, one row of stamps per
+    // phase: 0 producer starts, 1 first operands have landed, 2 last MMA issued, 3 last accumulator
+    // complete, 4 epilogues done, 5 grid barrier passed
+    int phase_no = 0;
+    __device__ void trace(int slot) const
+    {
+        if (r.trace == nullptr || phase_no >= JS_TRACE_PHASES) return;
+        if (blockIdx.x != 0 && blockIdx.x != gridDim.x - 1) return;
+        const int who = blockIdx.x == 0 ? 0 : 1;
+        r.trace[((size_t)who * JS_TRACE_PHASES + phase_no) * JS_TRACE_SLOTS + slot] = global_ns();
+    }
+
     __device__ bool barrier()
     {
         fence_proxy_async();      // epilogue stores are read by the next layer's TMA loads
         const bool ok = grid_barrier(r.ctl, epoch, r.spin_limit);
         fence_proxy_async();
+        if (threadIdx.x == 0) trace(5);
         return ok;
     }
 
@@ -172,6 +185,7 @@ struct ConvEngine {
         const CUtensorMap *ma = m.tmAct + l, *mw = m.tmW + l;
         const uint32_t bytes = A_BYTES + bn * BK * 2;
         const int kcs = head ? m.ch / BK : m.cin_pad[l] / BK;
+        trace(0);
         for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
             int n, yt, c;
             locate(id, nyl, yt_lo, per, n, yt, c);
@@ -203,6 +217,7 @@ struct ConvEngine {
             for (int kb = 0; kb < nkb; ++kb) {
                 if (!mbar_wait(&sh.full[stage], sphase, r.ctl)) { dead = true; break; }
                 tc_fence_after();
+                if (kb == 0 && id == (int)blockIdx.x) trace(1);
                 const uint64_t adesc = smem_desc_sw128(smem_u32(stage_a(stage)));
                 const uint64_t bdesc = smem_desc_sw128(smem_u32(stage_b(stage)));
 #pragma unroll
@@ -216,6 +231,7 @@ struct ConvEngine {
             umma_commit(&sh.tfull[acc]);
             advance_acc();
         }
+        trace(2);
     }
 
     __device__ void release_acc()
@@ -283,6 +299,7 @@ struct ConvEngine {
             }
             if (!mbar_wait(&sh.tfull[acc], aphase, r.ctl)) { dead = true; break; }
             tc_fence_after();
+            if (warp == 4 && lane == 0) trace(3);
             const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS);
             if (!head) {
                 epi_hidden_tile(l, n, y0, tbase);
@@ -299,6 +316,7 @@ struct ConvEngine {
                 int bi = 0;
                 for (int c0 = 0; c0 < 256; c0 += 32) {
                     float v[32];
+                    __syncwarp();
                     tmem_ld32(tbase + (uint32_t)c0, v);
                     if (!valid) continue;
                     if (kind == EPI_LOGITS) {
@@ -319,23 +337,34 @@ struct ConvEngine {
                         }
                     }
                 }
+                bool ch = false;
                 if (kind == EPI_CAT && valid && t >= w.plo && t < w.phi) {
                     if ((int)r.x[at] != bi) {
                         r.x[at] = (uint8_t)bi;
                         ((__nv_bfloat16 *)m.act[0])[((size_t)n * m.height * m.width + pix) * 64 + c] =
                             __float2bfloat16_rn(m.lut[bi]);
-                        if (flag) {
-                            int *f = &r.smp_changed[parity * r.batch + n];     // look first: stores to one
-                            if (ld_volatile_i32(f) == 0) *f = 1;                 // address serialise in L2
-                            any_changed = true;
-                            first = min(first, t);
-                        }
+                        ch = true;
+                    }
+                }
+                __syncwarp();
+                if (flag) {
+                    // every pixel of the tile belongs to image n: one lane reports for the warp, and it
+                    // looks before it stores (accesses to one address serialise in L2, and in the first
+                    // passes every pixel of every tile changes)
+                    if (__any_sync(0xffffffffu, ch) && lane == 0) {
+                        int *f = &r.smp_changed[parity * r.batch + n];
+                        if (ld_volatile_i32(f) == 0) *f = 1;
+                    }
+                    if (ch) {
+                        any_changed = true;
+                        first = min(first, t);
                     }
                 }
                 release_acc();
             }
             advance_acc();
         }
+        if (warp == 4 && lane == 0) trace(4);
         if (flag) {
             const bool wany = __any_sync(0xffffffffu, any_changed);
             if (wany) {
@@ -360,6 +389,7 @@ struct ConvEngine {
             if (blockIdx.x == 0) skipped += (unsigned long long)(r.batch * m.nyt - sh.n_img * nyl) * (head ? m.in_ch : 1);
         }
         if (ntiles == 0) return false;
+        phase_no++;
         if (warp == 0) {
             if (lane == 0) producer(l, yt_lo, nyl, ntiles);
         } else if (warp == 1) {
