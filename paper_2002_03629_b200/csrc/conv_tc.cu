@@ -42,6 +42,7 @@ struct ConvShared {
     uint64_t full[N_STAGES], empty[N_STAGES], tfull[2], tempty[2];
     uint32_t tmem_base;
     float bias_s[4][256];
+    float lut_s[256];         // input encoding table
     int img[MAX_IMAGES];      // images still iterating
     int n_img;
 };
@@ -73,6 +74,7 @@ struct ConvEngine {
     // phase: 0 producer starts, 1 first operands have landed, 2 last MMA issued, 3 last accumulator
     // complete, 4 epilogues done, 5 grid barrier passed
     int phase_no = 0;
+    int raised_img = -1, raised_phase = -1;      // last (image, phase) this warp reported a change for
     __device__ void trace(int slot) const
     {
         if (r.trace == nullptr || phase_no >= JS_TRACE_PHASES) return;
@@ -314,6 +316,10 @@ struct ConvEngine {
                 const float *bias = m.bias[m.n_conv] + (size_t)c * 256;
                 float best = -INFINITY;
                 int bi = 0;
+                // the current symbol, asked for now: its latency passes while the classes are reduced
+                const bool commit = kind == EPI_CAT && valid && t >= w.plo && t < w.phi;
+                int xold = 0;
+                if (commit) xold = (int)__ldcg(r.x + at);
                 for (int c0 = 0; c0 < 256; c0 += 32) {
                     float v[32];
                     __syncwarp();
@@ -324,43 +330,41 @@ struct ConvEngine {
                         for (int i = 0; i < 32; ++i) zout[at * 256 + c0 + i] = v[i] + bias[c0 + i];
                     } else {
                         const float *gg = r.noise + at * 256 + c0;
+                        float sc[32];
 #pragma unroll
                         for (int i = 0; i < 32; i += 4) {
                             const float4 b4 = __ldg(reinterpret_cast<const float4 *>(bias + c0 + i));
                             const float4 g4 = __ldg(reinterpret_cast<const float4 *>(gg + i));
-                            const float s0 = (v[i] + b4.x) + g4.x, s1 = (v[i + 1] + b4.y) + g4.y;
-                            const float s2 = (v[i + 2] + b4.z) + g4.z, s3 = (v[i + 3] + b4.w) + g4.w;
-                            if (s0 > best) { best = s0; bi = c0 + i; }
-                            if (s1 > best) { best = s1; bi = c0 + i + 1; }
-                            if (s2 > best) { best = s2; bi = c0 + i + 2; }
-                            if (s3 > best) { best = s3; bi = c0 + i + 3; }
+                            sc[i] = (v[i] + b4.x) + g4.x;
+                            sc[i + 1] = (v[i + 1] + b4.y) + g4.y;
+                            sc[i + 2] = (v[i + 2] + b4.z) + g4.z;
+                            sc[i + 3] = (v[i + 3] + b4.w) + g4.w;
                         }
+                        argmax_chunk32(sc, c0, best, bi);
                     }
                 }
+                release_acc();        // the accumulator has been read: the next tile's MMAs may have it
                 bool ch = false;
-                if (kind == EPI_CAT && valid && t >= w.plo && t < w.phi) {
-                    if ((int)r.x[at] != bi) {
-                        r.x[at] = (uint8_t)bi;
-                        ((__nv_bfloat16 *)m.act[0])[((size_t)n * m.height * m.width + pix) * 64 + c] =
-                            __float2bfloat16_rn(m.lut[bi]);
-                        ch = true;
-                    }
+                if (commit && xold != bi) {
+                    r.x[at] = (uint8_t)bi;
+                    ((__nv_bfloat16 *)m.act[0])[((size_t)n * m.height * m.width + pix) * 64 + c] =
+                        __float2bfloat16_rn(sh.lut_s[bi]);
+                    ch = true;
                 }
-                __syncwarp();
                 if (flag) {
-                    // every pixel of the tile belongs to image n: one lane reports for the warp, and it
-                    // looks before it stores (accesses to one address serialise in L2, and in the first
-                    // passes every pixel of every tile changes)
-                    if (__any_sync(0xffffffffu, ch) && lane == 0) {
-                        int *f = &r.smp_changed[parity * r.batch + n];
-                        if (ld_volatile_i32(f) == 0) *f = 1;
+                    // every pixel of the tile belongs to image n: one lane reports for the warp, with a
+                    // plain store (a load to look first would be an L2 round trip per tile), and only
+                    // once per image and phase
+                    if (__any_sync(0xffffffffu, ch) && (raised_img != n || raised_phase != phase_no)) {
+                        if (lane == 0) r.smp_changed[parity * r.batch + n] = 1;
+                        raised_img = n;
+                        raised_phase = phase_no;
                     }
                     if (ch) {
                         any_changed = true;
                         first = min(first, t);
                     }
                 }
-                release_acc();
             }
             advance_acc();
         }
@@ -425,6 +429,7 @@ conv_tc_kernel(const __grid_constant__ ConvDev m, const __grid_constant__ RunArg
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
+    for (int i = threadIdx.x; i < 256; i += blockDim.x) sh.lut_s[i] = m.lut[i];
     if (warp == 1) tmem_alloc(&sh.tmem_base, 512);
     tc_fence_before();
     __syncthreads();

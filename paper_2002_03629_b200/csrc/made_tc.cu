@@ -52,6 +52,7 @@ struct TcShared {
     uint64_t nzbar[4];             // per epilogue warp: bulk copies of a binary tile's noise and symbols
     uint32_t tmem_base;
     int off[JS_MAXL + 1];          // start of layer l's tile metadata inside `meta`
+    float lut_s[256];              // input encoding table (a lookup per committed symbol would be an L2 round trip)
     alignas(16) float bias_s[4][256];   // per epilogue warp: bias of the current tile's columns (read as float4)
     int wcnt[NTH / 32];            // compaction: per-warp counts
     int cbase;                     // compaction: rows kept so far
@@ -575,12 +576,19 @@ struct TcEngine {
         }
     }
 
-    // raise the per-sample change flag without hammering it: thousands of tiles report on the same
-    // few words, and stores to one address serialise in L2, so look first and store only if needed
+    // Raise the per-sample change flag.  Thousands of tiles report on the same few words, and
+    // accesses to one address serialise in L2; a load to look first would put an L2 round trip at
+    // the end of every tile's epilogue.  So: a plain store, and each thread remembers the last
+    // (sample, phase) it raised, which keeps it to one store per row and phase in the common case
+    // of a thread that meets the same row in tile after tile.
+    int raised_sample = -1;
+    unsigned raised_stamp = 0;
     __device__ void raise_flag(int parity, int sample)
     {
-        int *f = &r.smp_changed[parity * r.batch + sample];
-        if (ld_volatile_i32(f) == 0) *f = 1;
+        if (raised_sample == sample && raised_stamp == stamp) return;
+        r.smp_changed[parity * r.batch + sample] = 1;
+        raised_sample = sample;
+        raised_stamp = stamp;
     }
 
     // ---- binary output layer (128 positions per tile), thread = one sample row of the tile.
@@ -630,15 +638,15 @@ struct TcEngine {
     {
         const float *bs = sh.bias_s[warp - 2];
         uint8_t *nz = nz_row(), *xs = xs_row();
-        const float lut0 = m.lut[0], lut1 = m.lut[1];
+        const float lut0 = sh.lut_s[0], lut1 = sh.lut_s[1];
         // columns [clo, chi) of the tile are sampled; the others keep their symbol
         const int clo = max(w.plo - n0, 0), chi = min(min(w.phi, m.T) - n0, ncols);
         if (t.bin_bulk) {
             if (!mbar_wait(&sh.nzbar[warp & 3], nzphase, r.ctl)) return false;
             nzphase ^= 1u;
         }
-        uint32_t diff_any = 0;
-        int first = INT_MAX;
+        uint32_t diff_any = 0, fdiff = 0;
+        int fword = INT_MAX;
         const bool tr = (warp == 4 && lane == 0);
         if (tr) trace(6);
 #pragma unroll 1
@@ -681,7 +689,10 @@ struct TcEngine {
                         enc[k] = nv ? lut1 : lut0;
                     }
                     const uint32_t df = nw ^ xw;
-                    if (df != 0u && first == INT_MAX) first = n0 + c + ((__ffs((int)df) - 1) >> 3);
+                    // first word with a change and its difference, by selects; the position follows below
+                    const bool newfirst = df != 0u && fword == INT_MAX;
+                    fword = newfirst ? c : fword;
+                    fdiff = newfirst ? df : fdiff;
                     diff_any |= df;
                     xn[i] = nw;
                     en[i] = make_uint2(pack_bf16x2(enc[0], enc[1]), pack_bf16x2(enc[2], enc[3]));
@@ -698,6 +709,7 @@ struct TcEngine {
         __syncwarp();
         if (tr) trace(7);
         const bool changed = diff_any != 0u;
+        const int first = changed ? n0 + fword + ((__ffs((int)fdiff) - 1) >> 3) : INT_MAX;
         if (t.bin_bulk) {
             fence_proxy_async_smem();         // the rows were written through the generic proxy
             if (changed) {
@@ -764,6 +776,10 @@ struct TcEngine {
         }
         float best = -INFINITY;
         int bi = 0;
+        // the current symbol, asked for now: its latency passes while the classes are reduced
+        const bool commit = sample >= 0 && d >= w.plo && d < w.phi;
+        int xold = 0;
+        if (commit) xold = (int)__ldcg(r.x + (size_t)sample * m.T + d);
         float4 g4[8], gn[8];
         if (sample >= 0 && !smem_rows) {
 #pragma unroll
@@ -787,18 +803,16 @@ struct TcEngine {
             if (c0 == 256 - 32) release_acc();
             if (cur_parts > 0) add_partials(ra, c0);
             if (sample >= 0) {
+                float sc[32];
 #pragma unroll
                 for (int i = 0; i < 8; ++i) {
                     const float4 b4 = *reinterpret_cast<const float4 *>(bs + c0 + i * 4);
-                    const float s0 = (__uint_as_float(ra[4 * i]) + b4.x) + g4[i].x;
-                    const float s1 = (__uint_as_float(ra[4 * i + 1]) + b4.y) + g4[i].y;
-                    const float s2 = (__uint_as_float(ra[4 * i + 2]) + b4.z) + g4[i].z;
-                    const float s3 = (__uint_as_float(ra[4 * i + 3]) + b4.w) + g4[i].w;
-                    if (s0 > best) { best = s0; bi = c0 + 4 * i; }
-                    if (s1 > best) { best = s1; bi = c0 + 4 * i + 1; }
-                    if (s2 > best) { best = s2; bi = c0 + 4 * i + 2; }
-                    if (s3 > best) { best = s3; bi = c0 + 4 * i + 3; }
+                    sc[4 * i] = (__uint_as_float(ra[4 * i]) + b4.x) + g4[i].x;
+                    sc[4 * i + 1] = (__uint_as_float(ra[4 * i + 1]) + b4.y) + g4[i].y;
+                    sc[4 * i + 2] = (__uint_as_float(ra[4 * i + 2]) + b4.z) + g4[i].z;
+                    sc[4 * i + 3] = (__uint_as_float(ra[4 * i + 3]) + b4.w) + g4[i].w;
                 }
+                argmax_chunk32(sc, c0, best, bi);
                 if (!smem_rows) {
 #pragma unroll
                     for (int i = 0; i < 8; ++i) g4[i] = gn[i];
@@ -806,13 +820,10 @@ struct TcEngine {
             }
         }
         bool ch = false;
-        if (sample >= 0 && d >= w.plo && d < w.phi) {
-            const size_t at = (size_t)sample * m.T + d;
-            if ((int)__ldcg(r.x + at) != bi) {
-                r.x[at] = (uint8_t)bi;
-                ((__nv_bfloat16 *)m.a[0])[(size_t)row * m.T + d] = __float2bfloat16_rn(m.lut[bi]);
-                ch = true;
-            }
+        if (commit && xold != bi) {
+            r.x[(size_t)sample * m.T + d] = (uint8_t)bi;
+            ((__nv_bfloat16 *)m.a[0])[(size_t)row * m.T + d] = __float2bfloat16_rn(sh.lut_s[bi]);
+            ch = true;
         }
         if (flag && ch) {
             raise_flag(parity, sample);
@@ -998,6 +1009,7 @@ made_tc_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ TcDev 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
+    for (int i = threadIdx.x; i < (m.C == 1 ? 2 : m.C) && i < 256; i += blockDim.x) sh.lut_s[i] = m.lut[i];
     if (warp == 1) tmem_alloc(&sh.tmem_base, 512);
     // tile metadata of every layer into shared memory (the range searches and the K-loop bounds
     // would otherwise be chains of dependent global loads in every phase)

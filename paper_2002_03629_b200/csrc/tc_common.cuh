@@ -230,6 +230,28 @@ __device__ __forceinline__ float tc_act_fn(int act, float v)
     return __fdividef(v, 1.0f + __expf(-y2));
 }
 
+// Running argmax over chunks of 32 values, lowest index first among equals, without a branch per
+// value: the chunk's maximum by a tree of max operations, the lowest position that holds it by a
+// chain of selects, and one update of the running pair per chunk.  (A compare-and-branch per value
+// diverges in nearly every warp and made a 256-way argmax cost 4.5 us per tile.)
+__device__ __forceinline__ void argmax_chunk32(const float (&s)[32], int c0, float &best, int &bi)
+{
+    float t[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) t[i] = fmaxf(s[i], s[i + 16]);
+#pragma unroll
+    for (int w = 8; w >= 1; w >>= 1)
+#pragma unroll
+        for (int i = 0; i < w; ++i) t[i] = fmaxf(t[i], t[i + w]);
+    const float mx = t[0];
+    int idx = 31;
+#pragma unroll
+    for (int i = 30; i >= 0; --i) idx = (s[i] == mx) ? i : idx;
+    const bool upd = mx > best;
+    best = upd ? mx : best;
+    bi = upd ? c0 + idx : bi;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
 {
     __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);
