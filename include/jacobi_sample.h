@@ -36,7 +36,8 @@ extern "C" {
 
 typedef struct js_model js_model;   /* opaque; library-owned device memory */
 
-/* solver selection; block_hybrid(B) of the benchmark spec is JS_GS_JACOBI */
+/* solver selection; the block hybrid with blocks in order and Jacobi inside (Algorithm 3) is
+ * JS_GS_JACOBI, the one with all blocks in parallel and a sweep inside (Algorithm 2) JS_JACOBI_GS */
 typedef enum { JS_JACOBI = 0, JS_GAUSS_SEIDEL = 1, JS_GS_JACOBI = 2, JS_JACOBI_GS = 3 } js_mode;
 
 /* how u_t turns the conditional's logits z_t into x_t (Appendix A.3):
@@ -195,15 +196,21 @@ const char *js_last_cuda_error(void);   /* text of the last failed CUDA call on 
  * kernel needs is one fixed device array inside the library, js_noalloc_scratch_limit()
  * bytes (4 MiB), which every GPU that loads the library holds until the process exits.
  * A shape whose scratch (js_noalloc_scratch_needed) exceeds it is rejected with JS_ERR_ARG
- * and a message in js_noalloc_last_error().  The call makes no cudaMalloc/cudaFree and calls
- * no allocating library routine.
+ * and a message in js_noalloc_last_error().  The call itself makes no cudaMalloc/cudaFree
+ * and calls no allocating library routine.
  *
  * All calls share the one array and find the previous call's contents in it; the kernel
  * clears what must start at zero.  Calls that overlap on the GPU race on it: serialise them.
  * The first call on each device looks up the array's device address (with that device
- * current), so make it before any stream capture begins.  Runs on one CTA: meant for small
- * models.  Results equal jacobi_sample(..., JS_JACOBI, ...) on the same fp32 model: same
- * samples, same out_iters, same return codes (0, JS_NOT_CONVERGED, negative on error).
+ * current); it is also the call on which the driver loads this library's device code and
+ * the array onto that GPU, which may take the driver's allocator once.  So make one warm-up
+ * call per device at start-up, before the phase that must not allocate and before any
+ * stream capture begins.  The array of the CURRENT device serves the call: cuda_stream must
+ * belong to that device.  Every call copies a status word back and synchronises cuda_stream
+ * before it returns.  Runs on one CTA: meant for small models.  Results equal
+ * jacobi_sample(..., JS_JACOBI, ...) on the same fp32 model: same samples, same out_iters,
+ * same return codes (0, JS_NOT_CONVERGED, negative on error).  A position whose scores are
+ * all NaN or -inf gets class 0.
  */
 typedef struct {
     int T, C, L;

@@ -21,7 +21,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "jacobi_oracle.c")
 _LIB = os.path.join(_HERE, "libjacobi_oracle.so")
 
-NOISE_UNIFORM_ICDF, NOISE_LOGISTIC, NOISE_GUMBEL = 0, 1, 2
+NOISE_UNIFORM_ICDF, NOISE_LOGISTIC, NOISE_GUMBEL, NOISE_UNIFORM_CAT = 0, 1, 2, 3
 ACT_RELU, ACT_GELU_TANH = 0, 1
 PREC_F32, PREC_BF16 = 0, 1
 

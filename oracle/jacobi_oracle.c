@@ -27,7 +27,11 @@
  * 16-position binary model, the convergence propositions of Section 3, the
  * worked Examples 1-3 of Section 4.1 realised as hand-built networks, the
  * autoregressive property by bit flips, a hand-computed 3-position network,
- * and numpy re-computation of the forward pass.  Iteration counts on the
+ * numpy re-computation of the forward pass (default and caller-given degrees),
+ * the decision margins recomputed from the logits and checked by moving the
+ * noise just short of and just past them, and, for the categorical inverse
+ * CDF, enumeration of all outcomes of a 3-way model, its law by chi-square and
+ * exact boundary cases.  Iteration counts on the
  * random-weight workloads have no value in the paper to compare with:
  * "parity unpinned" for those counts (they are bounded by the propositions
  * and checked on Examples 1-3 only).
@@ -37,7 +41,7 @@
 #include <stdlib.h>
 #include <string.h>
 
-enum { ORC_NOISE_UNIFORM_ICDF = 0, ORC_NOISE_LOGISTIC = 1, ORC_NOISE_GUMBEL = 2 };
+enum { ORC_NOISE_UNIFORM_ICDF = 0, ORC_NOISE_LOGISTIC = 1, ORC_NOISE_GUMBEL = 2, ORC_NOISE_UNIFORM_CAT = 3 };
 enum { ORC_ACT_RELU = 0, ORC_ACT_GELU_TANH = 1 };
 enum { ORC_PREC_F32 = 0, ORC_PREC_BF16 = 1 };
 enum { ORC_KIND_MADE = 0, ORC_KIND_CONV = 1 };
@@ -124,7 +128,7 @@ orc_model *orc_made_create(int T, int C, int L, const int *H, int act, int prec,
                            const float *const *W, const float *const *b,
                            const float *lut, int n_lut, const int *const *hidden_deg)
 {
-    if (L < 1 || L > ORC_MAX_LAYERS || T < 1 || C < 1) return NULL;
+    if (L < 1 || L > ORC_MAX_LAYERS || T < 1 || C < 1 || C > 256) return NULL;
     orc_model *m = (orc_model *)calloc(1, sizeof(orc_model));
     m->kind = ORC_KIND_MADE; m->T = T; m->C = C; m->L = L; m->act = act; m->prec = prec;
     m->n_lut = n_lut;
@@ -211,10 +215,32 @@ static void made_forward(const orc_model *m, const uint8_t *x, float *z)
  *   UNIFORM_ICDF  x = [u < sigmoid(z)]             (inverse-CDF for a Bernoulli)
  *   LOGISTIC      x = [z + eps > 0]                (eps logistic: same law)
  *   GUMBEL        x = argmax_c (z_c + g_c), lowest index among equal maxima
+ *   UNIFORM_CAT   x = the first class c with u < F_c, F_c = sum_{i<=c} softmax(z)_i
+ *                 (inverse-CDF for a categorical: one uniform number per position)
  * nz: C logits of this position; noise: 1 value, or C values for GUMBEL.
  */
+
+/* unnormalised cumulative distribution of softmax(nz): cum[c] = sum_{i<=c} exp(nz[i] - max);
+ * returns the total cum[C-1] */
+static double softmax_cumulative(int C, const float *nz, double *cum)
+{
+    double mx = (double)nz[0];
+    for (int c = 1; c < C; ++c) if ((double)nz[c] > mx) mx = (double)nz[c];
+    double run = 0.0;
+    for (int c = 0; c < C; ++c) { run += exp((double)nz[c] - mx); cum[c] = run; }
+    return run;
+}
+
 static int sample_position(int C, const float *nz, const float *noise, int nk)
 {
+    if (nk == ORC_NOISE_UNIFORM_CAT) {
+        double cum[256];
+        double tot = softmax_cumulative(C, nz, cum);
+        double target = (double)noise[0] * tot;
+        for (int c = 0; c < C; ++c)
+            if (target < cum[c]) return c;
+        return C - 1;       /* u so close to 1 that rounding left it at the total */
+    }
     if (nk == ORC_NOISE_UNIFORM_ICDF) {
         float p = (float)(1.0 / (1.0 + exp(-(double)nz[0])));
         return noise[0] < p ? 1 : 0;
@@ -235,6 +261,20 @@ static int sample_position(int C, const float *nz, const float *noise, int nk)
 /* distance of the decision from a tie, in logit units */
 static float decision_margin(int C, const float *nz, const float *noise, int nk)
 {
+    if (nk == ORC_NOISE_UNIFORM_CAT) {
+        /* u lies between the cumulative probabilities F_{x-1} and F_x.  Moving every logit by at
+         * most d moves a cumulative probability by at most d/2, so twice the distance of u from
+         * the nearer boundary is the tie distance in logit units (the outermost boundaries 0
+         * and 1 do not move). */
+        double cum[256];
+        double tot = softmax_cumulative(C, nz, cum);
+        double u = (double)noise[0];
+        int x = sample_position(C, nz, noise, nk);
+        double gap = INFINITY;
+        if (x > 0) gap = u - cum[x - 1] / tot;
+        if (x < C - 1 && cum[x] / tot - u < gap) gap = cum[x] / tot - u;
+        return (float)(2.0 * gap);
+    }
     if (nk == ORC_NOISE_UNIFORM_ICDF) {
         double u = (double)noise[0];
         return (float)fabs((double)nz[0] - (log(u) - log1p(-u)));
@@ -308,7 +348,7 @@ orc_model *orc_conv_create(int height, int width, int in_ch, int ch, int n_conv,
                            const float *const *W, const float *const *b,
                            const float *lut, int n_lut)
 {
-    if (n_conv < 1 || n_conv > ORC_MAX_LAYERS) return NULL;
+    if (n_conv < 1 || n_conv > ORC_MAX_LAYERS || C < 1 || C > 256) return NULL;
     orc_model *m = (orc_model *)calloc(1, sizeof(orc_model));
     m->kind = ORC_KIND_CONV; m->height = height; m->width = width; m->in_ch = in_ch; m->ch = ch;
     m->n_conv = n_conv; m->C = C; m->T = height * width * in_ch; m->act = ORC_ACT_RELU; m->prec = prec;

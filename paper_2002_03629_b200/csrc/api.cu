@@ -107,6 +107,12 @@ int made_build(js_model *m, const js_made_desc *d)
     }
 
     // weights: upload unmasked fp32, mask and round on the device
+    int sms = 1;
+    {
+        int dev = 0;
+        CU_TRY(cudaGetDevice(&dev));
+        CU_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    }
     for (int l = 0; l <= L; ++l) {
         const size_t cnt = (size_t)v.n[l + 1] * v.n[l];
         float *tmp = nullptr;
@@ -116,7 +122,7 @@ int made_build(js_model *m, const js_made_desc *d)
         if (e == cudaSuccess) e = cudaMalloc(&wm, cnt * esz);
         if (e == cudaSuccess) {
             m->allocs.push_back(wm);
-            const int grid = (int)std::min<size_t>((cnt + 255) / 256, 148 * 16);
+            const int grid = (int)std::min<size_t>((cnt + 255) / 256, (size_t)sms * 16);
             if (d->prec == JS_BF16)
                 pack_made_weights<__nv_bfloat16><<<grid, 256>>>(tmp, v.deg[l + 1], v.deg[l], v.n[l + 1], v.n[l],
                                                                  l == L, (__nv_bfloat16 *)wm);
@@ -377,18 +383,33 @@ int jacobi_sample_host(const js_model *cm, int batch, const float *noise_host, i
     int rc = ensure_host_staging(m);
     if (rc != JS_OK) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream, cs = m->copy_stream;
+    // From the first enqueue on, every way out drains both streams first: the caller's buffers and
+    // the arrival word may only be touched during the call.
+    auto leave = [&](int code) {
+        cudaStreamSynchronize(cs);
+        cudaStreamSynchronize(st);
+        return code;
+    };
+#define HOST_TRY(call)                                                                       \
+    do {                                                                                     \
+        cudaError_t e__ = (call);                                                            \
+        if (e__ != cudaSuccess) {                                                            \
+            snprintf(g_cuda_err, sizeof g_cuda_err, "%s: %s", #call, cudaGetErrorString(e__)); \
+            return leave(JS_ERR_CUDA);                                                       \
+        }                                                                                    \
+    } while (0)
     // the uploads start once the work the caller queued on `st` before this call is done
-    CU_TRY(cudaEventRecord(m->ev_main, st));
-    CU_TRY(cudaStreamWaitEvent(cs, m->ev_main, 0));
+    HOST_TRY(cudaEventRecord(m->ev_main, st));
+    HOST_TRY(cudaStreamWaitEvent(cs, m->ev_main, 0));
     if (init_host) {
-        CU_TRY(cudaMemcpyAsync(m->st_init, init_host, (size_t)batch * T, cudaMemcpyHostToDevice, cs));
-        CU_TRY(cudaEventRecord(m->ev_copy, cs));
-        CU_TRY(cudaStreamWaitEvent(st, m->ev_copy, 0));       // the start iterate is needed at once
+        HOST_TRY(cudaMemcpyAsync(m->st_init, init_host, (size_t)batch * T, cudaMemcpyHostToDevice, cs));
+        HOST_TRY(cudaEventRecord(m->ev_copy, cs));
+        HOST_TRY(cudaStreamWaitEvent(st, m->ev_copy, 0));       // the start iterate is needed at once
     }
-    CU_TRY(cudaMemcpyAsync(m->st_noise, noise_host, (size_t)batch * T * C * sizeof(float), cudaMemcpyHostToDevice, cs));
+    HOST_TRY(cudaMemcpyAsync(m->st_noise, noise_host, (size_t)batch * T * C * sizeof(float), cudaMemcpyHostToDevice, cs));
     // copies of one stream run in order: this word changes after the noise has arrived
     *m->h_nflag = ++m->n_uploads;
-    CU_TRY(cudaMemcpyAsync(m->d_nflag, m->h_nflag, sizeof(unsigned), cudaMemcpyHostToDevice, cs));
+    HOST_TRY(cudaMemcpyAsync(m->d_nflag, m->h_nflag, sizeof(unsigned), cudaMemcpyHostToDevice, cs));
     RunArgs r;
     memset(&r, 0, sizeof r);
     r.batch = batch; r.noise = m->st_noise; r.nk = nk; r.init = init_host ? m->st_init : nullptr;
@@ -402,16 +423,17 @@ int jacobi_sample_host(const js_model *cm, int batch, const float *noise_host, i
         r.noise_ready = m->d_nflag;
         r.noise_stamp = m->n_uploads;
     } else {
-        CU_TRY(cudaEventRecord(m->ev_copy, cs));
-        CU_TRY(cudaStreamWaitEvent(st, m->ev_copy, 0));
+        HOST_TRY(cudaEventRecord(m->ev_copy, cs));
+        HOST_TRY(cudaStreamWaitEvent(st, m->ev_copy, 0));
     }
     rc = run_made(m, r, st);
-    CU_TRY(cudaStreamSynchronize(cs));
-    if (rc < 0) return rc;
-    CU_TRY(cudaMemcpyAsync(out_samples_host, m->st_x, (size_t)batch * T, cudaMemcpyDeviceToHost, st));
+    if (rc < 0) return leave(rc);
+    HOST_TRY(cudaStreamSynchronize(cs));
+    HOST_TRY(cudaMemcpyAsync(out_samples_host, m->st_x, (size_t)batch * T, cudaMemcpyDeviceToHost, st));
     if (out_iters_host)
-        CU_TRY(cudaMemcpyAsync(out_iters_host, m->st_iters, (size_t)batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
-    CU_TRY(cudaStreamSynchronize(st));
+        HOST_TRY(cudaMemcpyAsync(out_iters_host, m->st_iters, (size_t)batch * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    HOST_TRY(cudaStreamSynchronize(st));
+#undef HOST_TRY
     return rc;
 }
 

@@ -59,6 +59,7 @@ __device__ __forceinline__ void book_samples(const RunArgs &r, int parity, int k
             done[b] = 1;
             count[b] = add ? count[b] + k : k;
             if (final_write && r.out_iters) r.out_iters[b] = count[b];
+            atomicMax(&r.ctl->iters_max, count[b]);
         }
     }
 }

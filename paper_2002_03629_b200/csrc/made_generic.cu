@@ -172,6 +172,7 @@ __device__ void sample_phase(const MadeDev &m, const RunArgs &r, const float *z,
             const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
             if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
         }
+        if ((unsigned)bi >= (unsigned)C) bi = 0;      // no finite score in the row: class 0
         if (lane == 0 && bi != r.x[at]) {
             r.x[at] = (uint8_t)bi;
             a0[at] = from_f32<T>(m.lut[bi]);
@@ -317,6 +318,7 @@ __device__ void jgs_commit_phase(const MadeDev &m, const RunArgs &r, int j, int 
             const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
             if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
         }
+        if ((unsigned)bi >= (unsigned)C) bi = 0;
         if (lane == 0) {
             r.x[at] = (uint8_t)bi;
             ((T *)m.a[0])[at] = from_f32<T>(m.lut[bi]);

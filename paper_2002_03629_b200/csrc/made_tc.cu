@@ -19,8 +19,6 @@
 #include <cuda.h>
 
 #include <algorithm>
-#include <cstdio>
-#include <cstdlib>
 
 #include "js_common.cuh"
 #include "js_model.h"
@@ -1300,21 +1298,13 @@ int js_tc_prepare(js_model *mo)
                     // short, longest, next short, next longest ...; the middle of the sorted list comes last
                     v0 = mix;
                 }
-            std::vector<long long> load(G, 0);
             for (int c = 0; c < G; ++c) {
-                load[c] = finish(c, nullptr, 0);
                 off.push_back((int)flat.size());
                 for (const Item &it : lp[c]) flat.push_back(it.code);
                 for (const Item &it : lo0[c]) flat.push_back(it.code);
                 for (const Item &it : lo1[c]) flat.push_back(it.code);
             }
             off.push_back((int)flat.size());
-            if (getenv("JS_DEBUG_SCHED")) {
-                long long mx = 0, mn = 1 << 30;
-                for (int c = 0; c < G; ++c) { mx = std::max(mx, load[c]); mn = std::min(mn, load[c]); }
-                fprintf(stderr, "layer %d MT %d ch %d: G %d units %zu+%zu modelled finish min %lld max %lld\n", l, MT, ch, G,
-                        part.size(), own.size(), mn, mx);
-            }
         }
         auto up = [&](const std::vector<int> &h, const int **dst) -> bool {
             void *q = nullptr;

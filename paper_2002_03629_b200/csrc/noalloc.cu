@@ -21,8 +21,14 @@
 //     it; the kernel clears what has to start at zero.  Two calls that overlap
 //     on the GPU (different streams or threads) race on it: serialise them;
 //   * the first call on a device looks up the array's device address
-//     (cudaGetSymbolAddress, with that device current); make that first call
-//     before any stream capture begins.
+//     (cudaGetSymbolAddress, with that device current) and is the call that makes
+//     the driver load this library's device code and the array itself onto that
+//     GPU, so it may take the driver's allocator once: make one warm-up call per
+//     device at start-up, before the phase that must not allocate and before any
+//     stream capture begins.  The array that serves a call is the one of the
+//     CURRENT device; cuda_stream must belong to that device;
+//   * every call copies a status word back and synchronises cuda_stream before it
+//     returns.
 // The kernel is a single-CTA restatement of the CUDA-core sampler (same
 // accumulation order, same sampling rule), so its samples and iteration counts
 // equal jacobi_sample's in JS_JACOBI mode on the same fp32 model.
@@ -144,6 +150,7 @@ noalloc_jacobi_kernel(const NoallocNet net, unsigned char *scratch, int batch, c
                     const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
                     if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
                 }
+                if ((unsigned)bi >= (unsigned)C) bi = 0;      // no finite score in the row (NaN or -inf everywhere): class 0
                 if (lane == 0 && bi != x[i]) {
                     x[i] = (uint8_t)bi;
                     a[0][i] = net.lut[bi];

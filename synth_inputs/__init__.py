@@ -15,8 +15,9 @@ Recipe (all draws from ``numpy.random.Generator(PCG64(seed))``):
 * biases ``~ N(0, b_var)`` (zeros when ``b_var == 0``);
 * noise from 32 random bits ``r``: ``u = (r + 0.5) * 2**-32`` in float64, then
   logistic ``log(u) - log(1 - u)`` or Gumbel ``-log(-log(u))`` rounded to
-  float32; uniform noise uses 23 bits, ``(k + 0.5) * 2**-23``, which float32
-  holds exactly and which can never reach 0 or 1.
+  float32; uniform noise (one number per position, for binary and for C-way
+  inverse-CDF sampling alike) uses 23 bits, ``(k + 0.5) * 2**-23``, which
+  float32 holds exactly and which can never reach 0 or 1.
 """
 from __future__ import annotations
 
@@ -28,6 +29,7 @@ import numpy as np
 NOISE_UNIFORM_ICDF = 0
 NOISE_LOGISTIC = 1
 NOISE_GUMBEL = 2
+NOISE_UNIFORM_CAT = 3      # one uniform number per C-way position (inverse CDF of the softmax)
 
 ACT_RELU = 0
 ACT_GELU_TANH = 1
@@ -154,7 +156,7 @@ def draw_noise(cfg, batch: Optional[int] = None, salt: int = 0) -> np.ndarray:
     rng = _rng(cfg, 2, salt)
     shape = noise_shape(cfg, batch)
     r = rng.integers(0, 2 ** 32, size=shape, dtype=np.uint32)
-    if cfg.noise_kind == NOISE_UNIFORM_ICDF:
+    if cfg.noise_kind in (NOISE_UNIFORM_ICDF, NOISE_UNIFORM_CAT):
         k = (r >> np.uint32(9)).astype(np.float64)
         return ((k + 0.5) * 2.0 ** -23).astype(np.float32)
     u = (r.astype(np.float64) + 0.5) * 2.0 ** -32

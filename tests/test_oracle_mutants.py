@@ -27,6 +27,15 @@ MUTANTS = [
     ("conv keeps the tap to the right", "else if (ky == 1 && kx == 0) keep = 1;", "else if (ky == 1 && kx != 1) keep = 1;"),
     ("Jacobi cap one short", "int cap = (max_iters > 0 && max_iters < T) ? max_iters : T;", "int cap = (max_iters > 0 && max_iters < T) ? max_iters : T - 1;"),
     ("sweep starts units one degree late", "if (m->deg[l + 1][i] == t)", "if (m->deg[l + 1][i] == t - 1)"),
+    ("Gumbel margin always zero", "    return top - second;", "    return 0.0f;"),
+    ("runner-up not kept when the top moves", "if (v > top) { second = top; top = v; }", "if (v > top) { top = v; }"),
+    ("logistic margin with the wrong sign", "return fabsf(nz[0] + noise[0]);", "return fabsf(nz[0] - noise[0]);"),
+    ("inverse-CDF margin measured to the far boundary", "cum[x] / tot - u < gap) gap", "cum[x] / tot - u > gap) gap"),
+    ("categorical inverse CDF not strict", "if (target < cum[c]) return c;", "if (target <= cum[c]) return c;"),
+    ("cumulative sum starts one class late", "for (int c = 0; c < C; ++c) { run += exp((double)nz[c] - mx); cum[c] = run; }",
+     "for (int c = 0; c < C; ++c) { cum[c] = run; run += exp((double)nz[c] - mx); }"),
+    ("softmax without the logits' scale", "run += exp((double)nz[c] - mx); cum[c] = run; }", "run += exp(0.5 * ((double)nz[c] - mx)); cum[c] = run; }"),
+    ("custom degrees ignored", "? hidden_deg[l - 1][j]", "? 1 + (int)(((long long)j * (T - 1)) / m->n[l])"),
 ]
 
 
