@@ -3,7 +3,9 @@
 
 One step = one ``jacobi_sample`` call (the whole hot path: every Jacobi
 iteration's masked forward pass, the fused sampling and compare, the device-side
-loop) over one batch of the seeded synthetic workload.  Prints ONE JSON line.
+loop) over one batch of the seeded synthetic workload.  Prints ONE JSON line: the
+headline workload (``--workload``, default the largest masked MLP) on top, and under
+``workloads`` every seeded config measured the same way in the same run.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--mode jacobi|gs_jacobi|jacobi_gs]
     python bench.py --impl reference ...      # the CPU oracle on a bounded sample of the same workload
@@ -76,15 +78,6 @@ def load_peaks():
         return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
                 "bf16_tflops_sustained": p["bf16_tflops_sustained"], "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
-
-
-def algorithmic_bytes_per_pass(cfg) -> float:
-    """Bytes one forward pass has to move at least: live weights once, noise, symbols in and out."""
-    live = live_macs_per_sample(cfg)
-    if cfg.kind == "conv":
-        live = live // (cfg.height * cfg.width)      # a conv weight serves every pixel
-    noise = cfg.batch * cfg.D * (cfg.C if cfg.noise_kind == si.NOISE_GUMBEL else 1) * 4
-    return 2.0 * live + noise + 2.0 * cfg.batch * cfg.D
 
 
 def recorded_traffic(workload: str):
@@ -232,25 +225,55 @@ def run_reference(args, cfg):
 
 
 # -------------------------------------------------------------------- our arm
-def run_ours(args, cfg):
+NOMINAL = {"bf16_tflops": 2250.0, "hbm_gbs": 7700.0}      # data-sheet figures, for context beside the measured peaks
+
+
+def roofline_of(cfg, stats, it_np, ms_launch, peaks):
+    """Roofline record of one call.  Algorithmic work counts only what the method needs: the live
+    (unmasked) multiply-accumulates of a forward pass for every sample that was still iterating in that
+    pass (the sum of the per-sample iteration counts), and for bytes the weight tiles the passes had to
+    stream (counted by the kernel: each tile once per pass, tiles behind the frontier not at all) plus
+    the noise and symbols of the samples still iterating."""
+    live = live_macs_per_sample(cfg)
+    sample_passes = int(it_np.sum())
+    flops = 2.0 * live * sample_passes
+    noise_per_sample = cfg.D * (cfg.C if cfg.noise_kind == si.NOISE_GUMBEL else 1) * 4
+    wbytes = float(stats.weight_bytes) if stats.weight_bytes > 0 else 2.0 * live * stats.iterations
+    nbytes = wbytes + (noise_per_sample + 2.0 * cfg.D) * sample_passes
+    kernel_name = "conv_tc_kernel" if cfg.kind == "conv" else ("made_tc_kernel" if stats.path == 0 else "made_generic_kernel")
+    ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    sec = ms_launch / 1e3
+    if flops / nbytes >= ridge:
+        achieved, peak = flops / sec / 1e12, peaks["bf16_tflops"]
+        r = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+             "peak_source": peaks["source"] + " burst bf16 (kernel timed alone)",
+             "frac_of_nominal": achieved / NOMINAL["bf16_tflops"],
+             "note": "2 x live (unmasked) MACs per sample x sum over samples of the passes each was still iterating in"}
+    else:
+        achieved, peak = nbytes / sec / 1e9, peaks["hbm_gbs"]
+        r = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+             "peak_source": peaks["source"] + " copy bandwidth",
+             "frac_of_nominal": achieved / NOMINAL["hbm_gbs"],
+             "note": "weight tiles streamed (device-counted, once per pass, frontier-skipped tiles excluded) + noise and "
+                     "symbols of the samples still iterating"}
+    r.update({"traffic": recorded_traffic(cfg.name), "kernel": kernel_name + " (one launch = all iterations of one call)",
+              "flops_per_launch": flops, "bytes_per_launch": nbytes, "ms_per_launch": ms_launch,
+              "sample_passes": sample_passes,
+              "frac_full_batch": (2.0 * live * cfg.batch * stats.iterations) / sec / 1e12 / peaks["bf16_tflops"],
+              "mma_issued_tflops": float(stats.mma_flops) / sec / 1e12 if stats.mma_flops > 0 else None,
+              "mma_issued_frac": float(stats.mma_flops) / sec / 1e12 / peaks["bf16_tflops"] if stats.mma_flops > 0 else None})
+    return r
+
+
+def measure_workload(pkg, cfg, inputs, mode_name, block, steps, warmup, world, rank, local, profile, seq, sample_clocks):
+    """Times one workload on this rank.  Returns (record, extras) where extras holds what the
+    headline line needs beside the record (clocks, arrays for the CPU leg)."""
     import torch
     import torch.distributed as dist
 
-    import __graft_entry__ as ge
-    ge.build()
-    import paper_2002_03629_b200 as pkg
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
-    W, b, lut, noise = make_inputs(cfg)
+    W, b, lut, noise = inputs
     model = pkg.Model.from_config(cfg, W, b, lut)
-    del W, b
-    nk, mode, block = cfg.noise_kind, MODES[args.mode], args.block
+    nk, mode = cfg.noise_kind, MODES[mode_name]
     h_noise = torch.from_numpy(noise).pin_memory()
     d_noise = h_noise.cuda()
     out = torch.empty((cfg.batch, cfg.D), dtype=torch.uint8, device="cuda")
@@ -267,26 +290,25 @@ def run_ours(args, cfg):
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(max(warmup, 3)):
         rc = step()
         if rc != 0:
-            raise RuntimeError(f"jacobi_sample returned {rc}")
+            raise RuntimeError(f"jacobi_sample returned {rc} on {cfg.name}")
     it_np = iters.cpu().numpy()
     stats = model.stats()
 
     # ---- device-resident timing: K steps, L2 flushed between them, CUDA events per step
     barrier()
-    sampler = ClockSampler(local) if rank == 0 else None
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    sampler = ClockSampler(local) if (rank == 0 and sample_clocks) else None
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     for s, e in ev:
         flush.zero_()
         s.record()
         step()
         e.record()
     barrier()
-    ms = [s.elapsed_time(e) for s, e in ev]
-    total_ms = float(sum(ms))
-    if sampler and not args.profile:
+    total_ms = float(sum(s.elapsed_time(e) for s, e in ev))
+    if sampler and not profile:
         # the timed region is milliseconds long: keep the same load running (untimed) until
         # nvidia-smi has had time to take a few samples of the clocks under it
         t_end = time.perf_counter() + 0.8
@@ -301,19 +323,19 @@ def run_ours(args, cfg):
         raise RuntimeError("jacobi_sample_host and jacobi_sample disagree")
     barrier()
     t_e2e = []
-    for _ in range(1 if args.profile else args.steps):
+    for _ in range(1 if profile else steps):
         flush.zero_()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         pkg.jacobi_sample_host(model, h_noise, nk, None, mode, block, 0, h_out)
         t_e2e.append(time.perf_counter() - t0)
-    e2e_s = float(sum(t_e2e)) * (args.steps / len(t_e2e))
+    e2e_s = float(sum(t_e2e)) * (steps / len(t_e2e))
 
-    # ---- the same kernels in strict sequential order (speedup denominators)
-    seq = {}
-    if args.seq and rank == 0 and not args.profile:
+    # ---- the same model in strict sequential order (speedup denominators)
+    seq_rec = {}
+    if seq and rank == 0 and not profile:
         for name, opt in (("seq_skip", 1), ("seq_full", 0)):
-            if name == "seq_full" and args.seq == "skip":
+            if name == "seq_full" and seq == "skip":
                 continue
             model.set_option(pkg.JS_OPT_SEQ_SKIP, opt)
             out2 = torch.empty_like(out)
@@ -324,78 +346,150 @@ def run_ours(args, cfg):
             pkg.sequential_sample(model, d_noise, nk, out2)
             e.record()
             torch.cuda.synchronize()
-            seq[name + "_ms"] = s.elapsed_time(e)
-            seq[name + "_matches_jacobi"] = bool(torch.equal(out2, out))
+            seq_rec[name + "_ms"] = s.elapsed_time(e)
+            seq_rec[name + "_us_per_position"] = 1e3 * seq_rec[name + "_ms"] / cfg.D
+            seq_rec[name + "_matches_jacobi"] = bool(torch.equal(out2, out))
         model.set_option(pkg.JS_OPT_SEQ_SKIP, 0)
 
     total_ms, e2e_s = max_over_ranks([total_ms, e2e_s], device="cuda")
+    ms_launch = total_ms / steps
+    peaks = load_peaks()
+    rec = {"ms_per_call": ms_launch, "samples_per_s": whole_job_rate(cfg.batch, steps, world, total_ms / 1e3),
+           "mode": mode_name, "block": block, "batch": cfg.batch,
+           "iters_per_sample": {"mean": float(it_np.mean()), "max": int(it_np.max()),
+                                "forward_passes": int(stats.iterations)},
+           "kernel_path": "tensor-core" if stats.path == 0 else "cuda-core",
+           "tiles": {"issued": int(stats.tiles_issued), "skipped": int(stats.tiles_skipped)},
+           "e2e": {"value": cfg.batch * steps * world / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h_noise.numel() * 4),
+                   "d2h_bytes_per_step": int(h_out.numel())}}
+    if stats.path == 0:
+        rec["roofline"] = roofline_of(cfg, stats, it_np, ms_launch, peaks)
+    else:
+        rec["roofline"] = "latency-bound (CUDA-core kernels, a few kFLOP per pass)"
+    if seq_rec:
+        rec["sequential_on_gpu"] = seq_rec
+        for k in ("seq_skip_ms", "seq_full_ms"):
+            if k in seq_rec:
+                rec["speedup_vs_" + k[:-3]] = seq_rec[k] / ms_launch
+    extras = {"clocks": clocks, "samples": out.cpu().numpy(), "iters": it_np, "steps": steps}
+    model.close()
+    del d_noise, flush
+    torch.cuda.empty_cache()
+    return rec, extras
+
+
+def cpu_leg(cfg, inputs, mode_name, block, n, gpu_samples, gpu_iters):
+    """The oracle, as it stands, on n samples of the workload: its rate, its iteration counts beside the
+    GPU's on the same samples, and how many of those samples differ from the GPU's anywhere."""
+    import oracle
+    oracle.build()
+    W, b, lut, noise = inputs
+    cores = os.cpu_count() or 1
+    orc = oracle.from_config(cfg, W, b, lut)
+    nk = cfg.noise_kind
+
+    def one(i):
+        if mode_name == "jacobi":
+            r = orc.jacobi(noise[i], nk)
+        elif mode_name == "gs_jacobi":
+            r = orc.gs_jacobi(noise[i], nk, block)
+        elif mode_name == "jacobi_gs":
+            r = orc.jacobi_gs(noise[i], nk, block)
+        else:
+            r = (orc.gauss_seidel(noise[i], nk), 1)
+        return r[0], r[1]
+    t0 = time.perf_counter()
+    res = orc.map_batch(one, n, cores)
+    dt = time.perf_counter() - t0
+    its = [r[1] for r in res]
+    differing = int(sum(1 for i, r in enumerate(res) if not np.array_equal(r[0], gpu_samples[i])))
+    return {"value": n / dt, "unit": UNIT, "cores": min(cores, n), "kind": "oracle",
+            "sample": f"{n} of {cfg.batch} samples, {mode_name}, {dt:.1f} s",
+            "iters_per_sample_mean": float(np.mean(its)),
+            "gpu_iters_mean_on_same_samples": float(gpu_iters[:n].mean()),
+            "samples_differing_from_gpu": differing}
+
+
+def oracle_sample_count(cfg, budget_s):
+    cores = os.cpu_count() or 1
+    per_sample_s = (14.0 if cfg.kind == "conv" else 4.0) * live_macs_per_sample(cfg) / 0.6e9
+    return int(min(cfg.batch, max(1, budget_s * cores / per_sample_s)))
+
+
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+
+    import __graft_entry__ as ge
+    ge.build()
+    import paper_2002_03629_b200 as pkg
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    steps = args.steps
+    inputs = make_inputs(cfg)
+    rec, ex = measure_workload(pkg, cfg, inputs, args.mode, args.block, steps, args.warmup, world, rank, local,
+                               args.profile, args.seq, True)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
-
-    peaks = load_peaks()
-    n_samples = cfg.batch * args.steps * world
-    value = whole_job_rate(cfg.batch, args.steps, world, total_ms / 1e3)
-    live = live_macs_per_sample(cfg)
-    flops_per_launch = 2.0 * live * cfg.batch * stats.iterations
-    ms_launch = total_ms / args.steps
-    bytes_per_launch = algorithmic_bytes_per_pass(cfg) * stats.iterations
     dtype = "bf16" if cfg.prec == si.PREC_BF16 else "f32"
-    kernel_name = "conv_tc_kernel" if cfg.kind == "conv" else ("made_tc_kernel" if stats.path == 0 else "made_generic_kernel")
-    # bound of the dominant kernel: by arithmetic intensity against the ridge of the measured peaks
-    ridge = peaks["bf16_tflops"] * 1e12 / (peaks["hbm_gbs"] * 1e9)
-    if flops_per_launch / bytes_per_launch >= ridge:
-        achieved = flops_per_launch / (ms_launch / 1e3) / 1e12
-        peak = peaks["bf16_tflops"]
-        roofline = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                    "peak_source": peaks["source"] + " burst bf16 (kernel timed alone)",
-                    "note": "live (unmasked) MACs x 2 x batch x forward passes executed"}
-    else:
-        achieved = bytes_per_launch / (ms_launch / 1e3) / 1e9
-        peak = peaks["hbm_gbs"]
-        roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                    "peak_source": peaks["source"] + " copy bandwidth",
-                    "note": "(live weights + noise + symbols) x forward passes executed; skipped tiles are not subtracted"}
-    roofline.update({"traffic": recorded_traffic(cfg.name), "kernel": kernel_name + " (one launch = all iterations of one call)",
-                     "flops_per_launch": flops_per_launch, "bytes_per_launch": bytes_per_launch,
-                     "ms_per_launch": ms_launch})
-
-    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_launch, "higher_is_better": True, "scaling": "weak",
+    roof = rec["roofline"]
+    if not isinstance(roof, dict):
+        roof = {"bound": "alu", "achieved": None, "peak": None, "unit": "TFLOP/s", "frac": None, "traffic": None, "note": roof}
+    line = {"metric": METRIC, "value": rec["samples_per_s"], "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": rec["ms_per_call"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": dtype, "data": "synthetic",
-            "config": {"workload": cfg.name, "mode": args.mode, "block": block, "batch": cfg.batch, "T": cfg.D,
+            "config": {"workload": cfg.name, "mode": args.mode, "block": args.block, "batch": cfg.batch, "T": cfg.D,
                        "C": cfg.C, "hidden": list(cfg.H) if cfg.kind == "made" else [cfg.ch] * cfg.layers,
                        "parallelism": f"replicas x{world}",
                        "l2": "256 MB written between timed steps (L2 flush)"},
-            "iters_per_sample": {"mean": float(it_np.mean()), "max": int(it_np.max()),
-                                 "forward_passes": int(stats.iterations)},
-            "kernel_path": "tensor-core" if stats.path == 0 else "cuda-core",
-            "tiles": {"issued": int(stats.tiles_issued), "skipped": int(stats.tiles_skipped)},
-            "roofline": roofline,
-            "e2e": {"value": n_samples / e2e_s, "unit": UNIT, "h2d_bytes_per_step": int(h_noise.numel() * 4),
-                    "d2h_bytes_per_step": int(h_out.numel())},
-            "gpu_launches": args.steps,
-            "clocks": clocks}
-    if seq:
-        line["sequential_on_gpu"] = seq
-        for k in ("seq_skip_ms", "seq_full_ms"):
-            if k in seq:
-                line["speedup_vs_" + k[:-3]] = seq[k] / ms_launch
+            "iters_per_sample": rec["iters_per_sample"],
+            "kernel_path": rec["kernel_path"],
+            "tiles": rec["tiles"],
+            "roofline": roof,
+            "e2e": rec["e2e"],
+            "gpu_launches": steps,
+            "clocks": ex["clocks"]}
+    for k in ("sequential_on_gpu", "speedup_vs_seq_skip", "speedup_vs_seq_full"):
+        if k in rec:
+            line[k] = rec[k]
 
     # ---- CPU baseline: the oracle on a bounded sample of the same workload
     if not args.no_cpu_baseline and not args.profile:
-        import oracle
-        oracle.build()
-        W, b, lut, noise2 = make_inputs(cfg)
-        cores = os.cpu_count() or 1
         n = min(cfg.batch, args.ref_samples)
-        dt, its = oracle_sample_time(cfg, W, b, lut, noise2, args.mode, block, n, cores)
-        line["cpu_baseline"] = {"value": n / dt, "unit": UNIT, "cores": min(cores, n), "kind": "oracle",
-                                "sample": f"{n} of {cfg.batch} samples, {args.mode}, {dt:.1f} s",
-                                "iters_per_sample_mean": float(np.mean(its))}
-        line["iters_per_sample"]["oracle_mean_on_sample"] = float(np.mean(its))
-        line["iters_per_sample"]["gpu_mean_on_same_samples"] = float(it_np[:n].mean())
+        line["cpu_baseline"] = cpu_leg(cfg, inputs, args.mode, args.block, n, ex["samples"], ex["iters"])
+        line["iters_per_sample"]["oracle_mean_on_sample"] = line["cpu_baseline"]["iters_per_sample_mean"]
+        line["iters_per_sample"]["gpu_mean_on_same_samples"] = line["cpu_baseline"]["gpu_iters_mean_on_same_samples"]
+
+    # ---- the other seeded configs, each measured the same way (fewer details), one GPU only
+    if args.all_workloads and world == 1 and not args.profile:
+        wl = {cfg.name: {k: v for k, v in rec.items()}}
+        if "cpu_baseline" in line:
+            wl[cfg.name]["oracle"] = {k: line["cpu_baseline"][k] for k in
+                                      ("sample", "iters_per_sample_mean", "gpu_iters_mean_on_same_samples",
+                                       "samples_differing_from_gpu")}
+        del ex, inputs
+        for name, other in si.CONFIGS.items():
+            if name == cfg.name:
+                continue
+            in2 = make_inputs(other)
+            r2, ex2 = measure_workload(pkg, other, in2, "jacobi", 0, max(steps, 10), args.warmup, 1, 0, local, False,
+                                       "skip", False)
+            if not args.no_cpu_baseline:
+                n2 = oracle_sample_count(other, 4.0)
+                c2 = cpu_leg(other, in2, "jacobi", 0, n2, ex2["samples"], ex2["iters"])
+                r2["oracle"] = {k: c2[k] for k in ("sample", "iters_per_sample_mean", "gpu_iters_mean_on_same_samples",
+                                                   "samples_differing_from_gpu")}
+            wl[name] = r2
+            del ex2, in2
+        line["workloads"] = wl
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -416,6 +510,8 @@ def main():
     ap.add_argument("--ref-samples", type=int, default=0,
                     help="samples per step of the CPU oracle (0: sized for roughly 15 s of CPU work)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--one-workload", dest="all_workloads", action="store_false",
+                    help="skip the `workloads` object (the other seeded configs measured beside the headline one)")
     ap.add_argument("--profile", action="store_true",
                     help="only the warm-up and the timed steps (for short runs under a profiler)")
     args = ap.parse_args()
@@ -426,8 +522,7 @@ def main():
         args.block = cfg.blocks[0] if cfg.blocks else 64
     if args.ref_samples <= 0:
         cores = os.cpu_count() or 1
-        per_sample_s = 4.0 * live_macs_per_sample(cfg) / 0.6e9          # a few forward passes at ~0.6 GMAC/s
-        args.ref_samples = int(min(cfg.batch, max(cores, 15.0 * cores / per_sample_s)))
+        args.ref_samples = max(min(cores, cfg.batch), oracle_sample_count(cfg, 15.0))
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

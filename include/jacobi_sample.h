@@ -150,7 +150,10 @@ int js_forward_logits(const js_model *m, int batch, const uint8_t *x_dev, float 
 
 typedef enum {
     JS_OPT_FRONTIER_SKIP = 0,  /* 1 (default): skip positions and hidden units already final (proof of Prop. 1) */
-    JS_OPT_SEQ_SKIP = 1,       /* 0 (default): sequential_sample recomputes everything each step; 1: only the band that changed */
+    JS_OPT_SEQ_SKIP = 1,       /* how sequential_sample and JS_GAUSS_SEIDEL walk the strict order.  0: a full forward pass per
+                                  position; 1: per position only the tiles of the band that changed; 2 (default): the cached
+                                  sweep, every hidden unit evaluated once (Section 4.2; binary bf16 masked MLPs with sorted
+                                  degrees - other models take 0) */
     JS_OPT_SPIN_LIMIT = 2,     /* polls before a device-side wait gives up (default 1<<22) */
     JS_OPT_PATH = 3,           /* 0 (default): tensor-core kernels where the model allows; 1: CUDA-core kernels only */
     JS_OPT_COMPACT = 4,        /* 1 (default): move finished samples out of the working batch */
@@ -160,7 +163,8 @@ int js_set_option(js_model *m, int option, int value);
 
 /* counters of the most recent sampling call on this model */
 typedef struct {
-    int iterations;            /* forward passes executed (micro-steps for Jacobi-GS) */
+    int iterations;            /* forward passes executed; outer iterations for Jacobi-GS on the tensor cores (micro-steps
+                                  on the CUDA-core kernels); 1 for the cached sweep */
     int batch_iters_max;       /* largest per-sample iteration count */
     int final_frontier;        /* leading positions known final when the loop ended */
     long long tiles_issued;    /* output tiles computed */
@@ -168,6 +172,8 @@ typedef struct {
     int path;                  /* 0 tensor-core kernels, 1 CUDA-core kernels */
     int status;                /* the call's return value */
     int compactions;           /* times finished samples were moved out of the working batch */
+    long long mma_flops;       /* tensor-core kernels: flops of the MMA instructions issued (tile padding included) */
+    long long weight_bytes;    /* tensor-core kernels: weight bytes the call had to stream (each weight tile counted once per pass) */
 } js_stats;
 int js_get_stats(const js_model *m, js_stats *out);
 

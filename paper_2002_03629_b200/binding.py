@@ -50,7 +50,7 @@ class _NoallocMade(C.Structure):
 class JsStats(C.Structure):
     _fields_ = [("iterations", C.c_int), ("batch_iters_max", C.c_int), ("final_frontier", C.c_int),
                 ("tiles_issued", C.c_longlong), ("tiles_skipped", C.c_longlong), ("path", C.c_int),
-                ("status", C.c_int), ("compactions", C.c_int)]
+                ("status", C.c_int), ("compactions", C.c_int), ("mma_flops", C.c_longlong), ("weight_bytes", C.c_longlong)]
 
 
 def load_library():

@@ -185,16 +185,17 @@ bool noise_kind_ok(const js_model *m, int nk)
     return false;
 }
 
-int run_made(js_model *m, RunArgs &r, cudaStream_t st)
+const int NOT_REPORTED = -1000000;
+
+// model-owned fields of the launch arguments; the control block is cleared if the last call left it dirty
+int prep_args(js_model *m, RunArgs &r, cudaStream_t st)
 {
-    const MadeDev &v = m->made;
-    if (m->kind == 1 && r.kmode == KM_JACOBI_GS) return JS_ERR_UNSUPPORTED;
     r.ctl = m->ctl;
     r.smp_changed = m->smp_changed;
     r.smp_state = m->smp_state;
     r.x_old = m->x_old;
     r.frontier_skip = m->opt_frontier_skip;
-    r.seq_skip = m->opt_seq_skip;
+    r.seq_skip = m->opt_seq_skip == 1 ? 1 : 0;
     r.compact = m->opt_compact;
     r.perm = m->perm;
     r.perm_stride = m->rows;
@@ -205,8 +206,146 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
     if (!m->ctl_clean) CU_TRY(cudaMemsetAsync(m->ctl, 0, sizeof(JsCtl), st));
     m->ctl_clean = false;
     r.result = m->d_result;
-    const int NOT_REPORTED = -1000000;
     m->h_result->status = NOT_REPORTED;
+    return JS_OK;
+}
+
+// waits for the launch and reads what the kernel reported through mapped host memory
+int wait_result(js_model *m, cudaStream_t st, JsCtl &h)
+{
+    CU_TRY(cudaStreamSynchronize(st));
+    h = *m->h_result;
+    if (h.status == NOT_REPORTED) {
+        snprintf(g_cuda_err, sizeof g_cuda_err, "the kernel ended without reporting");
+        return JS_ERR_CUDA;
+    }
+    m->ctl_clean = h.status >= 0;
+    return JS_OK;
+}
+
+int launch_failed(int rc_launch)
+{
+    snprintf(g_cuda_err, sizeof g_cuda_err, "kernel launch: %s", cudaGetErrorString((cudaError_t)rc_launch));
+    return JS_ERR_CUDA;
+}
+
+void fill_stats(js_model *m, const JsCtl &h, int used_path)
+{
+    m->stats.iterations = h.iterations;
+    m->stats.final_frontier = h.frontier;
+    m->stats.tiles_issued = (long long)h.tiles_issued;
+    m->stats.tiles_skipped = (long long)h.tiles_skipped;
+    m->stats.batch_iters_max = h.iters_max;
+    m->stats.mma_flops = (long long)h.mma_flops;
+    m->stats.weight_bytes = (long long)h.weight_bytes;
+    m->stats.path = used_path;
+    m->stats.compactions = h.compactions;
+    m->stats.status = h.status;
+}
+
+// can the cached sweeps (made_sweep.cu) serve this call?
+bool sweeps_usable(js_model *m, const RunArgs &r)
+{
+    if (m->kind != 0 || !m->tc_ok || m->opt_path != 0 || m->made.C != 1) return false;
+    if ((((uintptr_t)r.noise | (uintptr_t)r.x) & 15u) != 0) return false;
+    return js_sweep_prepare(m) == 1;
+}
+
+// The feedforward pass with every hidden unit evaluated once: one sweep over all positions.
+int run_sweep_sequential(js_model *m, RunArgs &r, cudaStream_t st)
+{
+    int rc = prep_args(m, r, st);
+    if (rc != JS_OK) return rc;
+    r.block = m->made.T;
+    r.blk_lo = 0;
+    r.smp_changed = m->sw_flags;
+    const int rl = js_launch_made_sweep(m, r, st);
+    if (rl != 0) return launch_failed(rl);
+    JsCtl h;
+    if ((rc = wait_result(m, st, h)) != JS_OK) return rc;
+    fill_stats(m, h, 0);
+    m->stats.iterations = 1;
+    m->stats.final_frontier = m->made.T;
+    if (h.status == JS_OK && r.out_iters) {
+        std::vector<int32_t> ones(r.batch, 1);
+        CU_TRY(cudaMemcpyAsync(r.out_iters, ones.data(), sizeof(int32_t) * r.batch, cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaStreamSynchronize(st));
+    }
+    return h.status;
+}
+
+// Algorithm 2 on the tensor cores.  Outer iteration k: the hidden layers on x^{k-1} (tensor-core
+// kernel, hidden layers only), then every block swept from that prefix (sweep kernel), then the
+// per-sample bookkeeping; the host looks at one word per outer iteration.  After k outer iterations
+// the first k blocks are final (proof of Proposition 2): they are not swept again, and the hidden
+// units that depend on them alone are not recomputed.
+int run_jacobi_gs_tc(js_model *m, RunArgs &r, cudaStream_t st)
+{
+    const MadeDev &v = m->made;
+    const int T = v.T, B = r.block, M = (T + B - 1) / B;
+    const int cap = (r.max_iters > 0 && r.max_iters < M) ? r.max_iters : M;
+    if (r.init != r.x) {
+        if (r.init) CU_TRY(cudaMemcpyAsync(r.x, r.init, (size_t)r.batch * T, cudaMemcpyDeviceToDevice, st));
+        else CU_TRY(cudaMemsetAsync(r.x, 0, (size_t)r.batch * T, st));
+    }
+    CU_TRY(cudaMemsetAsync(m->sw_flags, 0, 2 * (size_t)m->rows * sizeof(int), st));
+    long long flops = 0;
+    int status = JS_OK, k = 0;
+    for (k = 1;; ++k) {
+        const int fin_blocks = m->opt_frontier_skip ? k - 1 : 0;          // blocks known final before this iteration
+        RunArgs f = r;
+        int rc = prep_args(m, f, st);
+        if (rc != JS_OK) return rc;
+        f.kmode = KM_HIDDEN;
+        f.x_in = r.x;
+        f.x = nullptr;
+        f.out_iters = nullptr;
+        f.hid_lo = m->opt_frontier_skip ? std::max(0, (k - 2) * B) : 0;   // final since the previous forward pass
+        int rl = js_launch_made_tc(m, f, st);
+        if (rl != 0) return launch_failed(rl);
+        JsCtl h;
+        if ((rc = wait_result(m, st, h)) != JS_OK) return rc;
+        if (h.status < 0) { fill_stats(m, h, 0); return h.status; }
+        flops += (long long)h.mma_flops;
+        RunArgs s2 = r;
+        if ((rc = prep_args(m, s2, st)) != JS_OK) return rc;
+        s2.blk_lo = std::min(fin_blocks, M - 1);
+        s2.smp_changed = m->sw_flags;
+        rl = js_launch_made_sweep(m, s2, st);
+        if (rl != 0) return launch_failed(rl);
+        *m->h_any = -1;
+        rl = js_launch_jgs_book(m, r.batch, k, k == cap, r.out_iters, st);
+        if (rl != 0) return launch_failed(rl);
+        if ((rc = wait_result(m, st, h)) != JS_OK) return rc;
+        flops += (long long)h.mma_flops;
+        if (h.status < 0) { fill_stats(m, h, 0); return h.status; }
+        const int any = *m->h_any;
+        if (any < 0) {
+            snprintf(g_cuda_err, sizeof g_cuda_err, "the bookkeeping kernel did not report");
+            return JS_ERR_CUDA;
+        }
+        fill_stats(m, h, 0);
+        if (!any || k == cap) {
+            if (any && cap < M) status = JS_NOT_CONVERGED;
+            break;
+        }
+    }
+    m->stats.iterations = k;
+    m->stats.mma_flops = flops;
+    m->stats.final_frontier = status == JS_OK ? T : std::min(T, k * B);
+    m->stats.status = status;
+    return status;
+}
+
+int run_made(js_model *m, RunArgs &r, cudaStream_t st)
+{
+    const MadeDev &v = m->made;
+    if (m->kind == 1 && r.kmode == KM_JACOBI_GS) return JS_ERR_UNSUPPORTED;
+    // the sweeps: the strict order with cached hidden units, and Algorithm 2
+    if (r.kmode == KM_SEQ && m->opt_seq_skip == 2 && sweeps_usable(m, r)) return run_sweep_sequential(m, r, st);
+    if (r.kmode == KM_JACOBI_GS && sweeps_usable(m, r)) return run_jacobi_gs_tc(m, r, st);
+    int rc = prep_args(m, r, st);
+    if (rc != JS_OK) return rc;
 
     int used_path = 1;
     int rc_launch;
@@ -220,12 +359,11 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
         used_path = 0;
         rc_launch = js_launch_made_tc(m, r, st);
     } else {
-    if (m->max_grid_generic <= 0) m->max_grid_generic = js_made_generic_max_grid(v.prec);
-    if (m->max_grid_generic <= 0) {
-        snprintf(g_cuda_err, sizeof g_cuda_err, "occupancy query failed");
-        return JS_ERR_CUDA;
-    }
-    {
+        if (m->max_grid_generic <= 0) m->max_grid_generic = js_made_generic_max_grid(v.prec);
+        if (m->max_grid_generic <= 0) {
+            snprintf(g_cuda_err, sizeof g_cuda_err, "occupancy query failed");
+            return JS_ERR_CUDA;
+        }
         long long tiles = 1;
         for (int l = 0; l <= v.L; ++l)
             tiles = std::max<long long>(tiles, (long long)((r.batch + JS_GT - 1) / JS_GT) * ((v.n[l + 1] + JS_GT - 1) / JS_GT));
@@ -233,26 +371,10 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
         const int grid = (int)std::min<long long>(m->max_grid_generic, std::max(tiles, elems));
         rc_launch = js_launch_made_generic(v, r, std::max(grid, 1), st);
     }
-    }
-    if (rc_launch != 0) {
-        snprintf(g_cuda_err, sizeof g_cuda_err, "kernel launch: %s", cudaGetErrorString((cudaError_t)rc_launch));
-        return JS_ERR_CUDA;
-    }
-    CU_TRY(cudaStreamSynchronize(st));
-    const JsCtl h = *m->h_result;
-    if (h.status == NOT_REPORTED) {
-        snprintf(g_cuda_err, sizeof g_cuda_err, "the kernel ended without reporting");
-        return JS_ERR_CUDA;
-    }
-    m->ctl_clean = h.status >= 0;
-    m->stats.iterations = h.iterations;
-    m->stats.final_frontier = h.frontier;
-    m->stats.tiles_issued = (long long)h.tiles_issued;
-    m->stats.tiles_skipped = (long long)h.tiles_skipped;
-    m->stats.batch_iters_max = h.iters_max;
-    m->stats.path = used_path;
-    m->stats.compactions = h.compactions;
-    m->stats.status = h.status;
+    if (rc_launch != 0) return launch_failed(rc_launch);
+    JsCtl h;
+    if ((rc = wait_result(m, st, h)) != JS_OK) return rc;
+    fill_stats(m, h, used_path);
     return h.status;
 }
 
@@ -322,6 +444,7 @@ void js_model_destroy(js_model *m)
     for (void *p : m->allocs) cudaFree(p);
     if (m->h_result) cudaFreeHost(m->h_result);
     if (m->h_nflag) cudaFreeHost(m->h_nflag);
+    if (m->h_any) cudaFreeHost(m->h_any);
     if (m->ev_main) cudaEventDestroy(m->ev_main);
     if (m->ev_copy) cudaEventDestroy(m->ev_copy);
     if (m->copy_stream) cudaStreamDestroy(m->copy_stream);
@@ -418,7 +541,7 @@ int jacobi_sample_host(const js_model *cm, int batch, const float *noise_host, i
     r.block = block; r.max_iters = max_iters;
     r.x = m->st_x; r.out_iters = m->st_iters;
     // only the tensor-core kernel of the masked MLPs waits for the noise by itself
-    const bool overlap = m->kind == 0 && m->tc_ok && m->opt_path == 0 && r.kmode != KM_JACOBI_GS;
+    const bool overlap = m->kind == 0 && m->tc_ok && m->opt_path == 0 && (r.kmode == KM_JACOBI || r.kmode == KM_GS_JACOBI);
     if (overlap) {
         r.noise_ready = m->d_nflag;
         r.noise_stamp = m->n_uploads;
@@ -468,7 +591,7 @@ int js_set_option(js_model *m, int option, int value)
     if (!m) return JS_ERR_ARG;
     switch (option) {
     case JS_OPT_FRONTIER_SKIP: m->opt_frontier_skip = value ? 1 : 0; return JS_OK;
-    case JS_OPT_SEQ_SKIP: m->opt_seq_skip = value ? 1 : 0; return JS_OK;
+    case JS_OPT_SEQ_SKIP: if (value < 0 || value > 2) return JS_ERR_ARG; m->opt_seq_skip = value; return JS_OK;
     case JS_OPT_SPIN_LIMIT: if (value < 0) return JS_ERR_ARG; m->opt_spin_limit = value; return JS_OK;
     case JS_OPT_PATH: if (value != 0 && value != 1) return JS_ERR_ARG; m->opt_path = value; return JS_OK;
     case JS_OPT_COMPACT: m->opt_compact = value ? 1 : 0; return JS_OK;

@@ -54,7 +54,7 @@ struct ConvEngine {
     ConvShared &sh;
     uint8_t *ring, *staging;
     unsigned epoch = 0;
-    unsigned long long issued = 0, skipped = 0;
+    unsigned long long issued = 0, skipped = 0, mma_flops = 0, weight_bytes = 0;
     int warp, lane;
     int stage = 0;
     uint32_t sphase = 0;
@@ -389,7 +389,13 @@ struct ConvEngine {
         const int nyl = yt_hi - yt_lo;
         const int ntiles = sh.n_img * nyl * (head ? m.in_ch : 1);
         if (threadIdx.x == 0) {
-            for (int id = blockIdx.x; id < ntiles; id += gridDim.x) issued++;
+            for (int id = blockIdx.x; id < ntiles; id += gridDim.x) {
+                issued++;
+                mma_flops += 2ull * BM * BK * (unsigned long long)(head ? 256 : m.ch) * (unsigned long long)kblocks(l);
+            }
+            // a layer's packed weights serve every tile: the pass streams them once
+            if (blockIdx.x == 0 && ntiles > 0)
+                weight_bytes += 2ull * BK * (unsigned long long)kblocks(l) * (unsigned long long)(head ? 256 * m.in_ch : m.ch);
             if (blockIdx.x == 0) skipped += (unsigned long long)(r.batch * m.nyt - sh.n_img * nyl) * (head ? m.in_ch : 1);
         }
         if (ntiles == 0) return false;
@@ -451,7 +457,7 @@ conv_tc_kernel(const __grid_constant__ ConvDev m, const __grid_constant__ RunArg
         tc_fence_after();
         tmem_dealloc(e.tmem_base, 512);
     }
-    driver_finish(r, res, e.issued, e.skipped);
+    driver_finish(r, res, e.issued, e.skipped, e.mma_flops, e.weight_bytes);
 }
 
 }  // namespace

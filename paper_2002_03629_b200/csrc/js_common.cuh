@@ -13,7 +13,8 @@
 #define JS_TRACE_SLOTS 12
 #define JS_GT 64          // output-tile edge of the CUDA-core GEMM phases
 
-enum { KM_JACOBI = 0, KM_SEQ = 1, KM_GS_JACOBI = 2, KM_JACOBI_GS = 3, KM_FORWARD = 4 };
+enum { KM_JACOBI = 0, KM_SEQ = 1, KM_GS_JACOBI = 2, KM_JACOBI_GS = 3, KM_FORWARD = 4,
+       KM_HIDDEN = 5 };      // KM_HIDDEN: hidden layers only, on the symbols x_in (activations for the sweeps)
 
 // Control block in device memory, zeroed by the host before every launch.
 struct JsCtl {
@@ -28,6 +29,8 @@ struct JsCtl {
     int live;               // samples still iterating (tensor-core path)
     int compactions;        // times the working batch was compacted
     unsigned long long tiles_issued, tiles_skipped;
+    unsigned long long mma_flops;       // flops of the tcgen05.mma instructions issued (tile padding included)
+    unsigned long long weight_bytes;    // bytes of weight tiles loaded for the first row tile of every unit (unique weight bytes a pass streams)
     unsigned exit_count;    // CTAs that have left; the last one reports and clears the block
 };
 
@@ -65,6 +68,8 @@ struct RunArgs {
     int *perm;                // [2][perm_stride]: working row -> sample index, by compaction parity
     int perm_stride;
     int frontier_skip, seq_skip, compact;
+    int blk_lo;               // sweeps: first block that is swept (earlier ones are final)
+    int hid_lo;               // KM_HIDDEN: hidden units of degree <= hid_lo are final already
     unsigned spin_limit;
     JsCtl *ctl;
     const unsigned *noise_ready;   // NULL, or a word that takes the value noise_stamp once `noise` has arrived

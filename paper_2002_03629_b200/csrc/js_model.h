@@ -38,6 +38,18 @@ struct TcDev {
     int n_pflags;
 };
 
+// What the cached sweeps (made_sweep.cu) need beside the tensor-core view.
+struct SweepDev {
+    const CUtensorMap *tmAold;          // [L+1] activations a[l] of the previous iterate, box 64 x 128 (= TcDev::tmA)
+    const CUtensorMap *tmF;             // [L+1] the jobs' buffers F[l], 3-D {column, row, slot}, box 64 x 128 x 1
+    const CUtensorMap *tmW16;           // [L+1] masked weights W[l], box 64 x 16
+    __nv_bfloat16 *F[JS_MAXL + 1];      // [slot][128 rows][WF[l]]: a job's fresh activations of a[l]
+    int WF[JS_MAXL + 1];
+    const int *cnt[JS_MAXL + 1];        // cnt[l][d], d = 0..T: units of a[l] with degree <= d (l >= 1)
+    int G;                              // positions per group
+    int n_stages, smem_bytes, slots;
+};
+
 // Device view of a masked-convolution stack (tensor-core kernel only).
 struct ConvDev {
     int height, width, in_ch, ch, n_conv, C, T;
@@ -74,12 +86,16 @@ struct js_model {
     int *smp_changed = nullptr, *smp_state = nullptr, *perm = nullptr;
     uint8_t *x_old = nullptr, *x_tmp = nullptr;
     unsigned long long *trace = nullptr;
-    int opt_frontier_skip = 1, opt_seq_skip = 0, opt_spin_limit = 1 << 22, opt_path = 0, opt_compact = 1, opt_trace = 0;
+    int opt_frontier_skip = 1, opt_seq_skip = 2, opt_spin_limit = 1 << 22, opt_path = 0, opt_compact = 1, opt_trace = 0;
     int max_grid_generic = 0;
     TcDev tc{};
     int tc_ok = 0, tc_max_grid = 0;
     ConvDev conv{};
     int conv_max_grid = 0;
+    SweepDev sweep{};
+    int sweep_state = 0;          // 0 not prepared yet, 1 ready, -1 the model does not qualify
+    int *sw_flags = nullptr;      // [2][rows]: per-sample change flags and done flags of the sweeps
+    int *h_any = nullptr, *d_any = nullptr;      // mapped host word: did anything change in this outer iteration
     js_stats stats{};
 };
 
@@ -87,3 +103,6 @@ int js_tc_prepare(js_model *m);
 int js_launch_made_tc(const js_model *m, const RunArgs &r, cudaStream_t stream);
 int js_conv_build(js_model *m, const js_conv_desc *d);
 int js_launch_conv_tc(const js_model *m, const RunArgs &r, cudaStream_t stream);
+int js_sweep_prepare(js_model *m);
+int js_launch_made_sweep(const js_model *m, const RunArgs &r, cudaStream_t stream);
+int js_launch_jgs_book(const js_model *m, int batch, int k, int at_cap, int32_t *out_iters, cudaStream_t stream);

@@ -111,12 +111,12 @@ __device__ DriverResult made_driver(E &e, int T_, const RunArgs &r)
         }
         return res;
     }
-    if (mode != KM_FORWARD && mode != KM_SEQ && mode != KM_JACOBI && mode != KM_GS_JACOBI) {
+    if (mode != KM_FORWARD && mode != KM_HIDDEN && mode != KM_SEQ && mode != KM_JACOBI && mode != KM_GS_JACOBI) {
         res.status = JS_ERR_ARG;
         return res;
     }
 
-    e.init(mode == KM_FORWARD ? r.x_in : mode == KM_SEQ ? (const uint8_t *)nullptr : r.init);
+    e.init((mode == KM_FORWARD || mode == KM_HIDDEN) ? r.x_in : mode == KM_SEQ ? (const uint8_t *)nullptr : r.init);
     if (!e.barrier()) { res.alive = false; return res; }
 
     // state shared by the modes
@@ -134,6 +134,8 @@ __device__ DriverResult made_driver(E &e, int T_, const RunArgs &r)
         if (mode == KM_FORWARD) {
             w = make_win(0, T_, 0, T_);
             zout = r.logits_out;
+        } else if (mode == KM_HIDDEN) {
+            w = make_win(r.hid_lo, T_, 0, 0);               // no output position: the hidden layers alone
         } else if (mode == KM_SEQ) {
             // Eq. 1 in strict order: step a keeps position a of a forward pass
             w = make_win(0, T_, a, a + 1);
@@ -151,7 +153,7 @@ __device__ DriverResult made_driver(E &e, int T_, const RunArgs &r)
         if (!e.step(w, flag, p, zout)) { res.alive = false; return res; }
         res.iterations++;
 
-        if (mode == KM_FORWARD) break;
+        if (mode == KM_FORWARD || mode == KM_HIDDEN) break;
         if (mode == KM_SEQ) {
             if (++a == T_) break;
             continue;
@@ -203,12 +205,15 @@ __device__ DriverResult made_driver(E &e, int T_, const RunArgs &r)
 // mapped host memory (so that the host needs no device-to-host copy) and zeroes it, ready for
 // the next launch (so that the host needs no memset either, unless a call ended abnormally).
 __device__ __forceinline__ void driver_finish(const RunArgs &r, const DriverResult &res, unsigned long long issued,
-                                              unsigned long long skipped)
+                                              unsigned long long skipped, unsigned long long mma_flops = 0,
+                                              unsigned long long weight_bytes = 0)
 {
     if (threadIdx.x != 0) return;
     JsCtl *c = r.ctl;
     atomicAdd(&c->tiles_issued, issued);
     atomicAdd(&c->tiles_skipped, skipped);
+    if (mma_flops) atomicAdd(&c->mma_flops, mma_flops);
+    if (weight_bytes) atomicAdd(&c->weight_bytes, weight_bytes);
     if (blockIdx.x == 0) {
         c->iterations = res.iterations;
         c->frontier = res.frontier;

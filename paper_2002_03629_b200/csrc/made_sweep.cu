@@ -1,0 +1,563 @@
+// Cached sequential sweeps of a masked MLP with binary positions, on the sm_100a tensor cores.
+//
+// A sweep computes positions a .. b-1 of a block strictly in order (Eq. 1 of arXiv 2002.03629),
+// each from the positions before it: positions < a are given (their hidden activations come from
+// a forward pass on the previous iterate), positions inside the block are the fresh ones.  That is
+// the inner loop of Jacobi-GS (Algorithm 2: all blocks in parallel, a sweep inside each) and, with
+// one block covering every position, the feedforward pass itself with every hidden unit evaluated
+// once (the cached sampler of Section 4.2).
+//
+// Work decomposition.  A job is (128 samples, one block); jobs never talk to each other, so the
+// kernel needs no grid-wide synchronisation at all.  Inside a job the positions are taken in
+// groups of G.  With sorted degrees, everything a group needs from before the group - inputs and
+// hidden units of degree <= t0, the group's first position - is a PREFIX of every layer's units,
+// so its contribution to the group's G output logits and to the handful of hidden units of degree
+// t0+1 .. t0+G is a GEMM  [128 samples x prefix] x [prefix x (<= 32 units)]  per layer: TMA feeds
+// the prefix of the activations (from the previous iterate's activations up to the block's start,
+// from the job's own buffer F after it) and 16-row weight boxes, tcgen05.mma accumulates in tensor
+// memory.  What the units of the group contribute to one another is a triangular system of at most
+// 32 x 32 weights per layer, solved position by position with thread = sample row: logit, sample
+// against the fixed noise (Appendix A.3), then the hidden units that the new symbol makes
+// computable.  The group's activations then go to F, where the next group's GEMMs find them.
+//
+// Every value is a fixed function of the iterate: the split into prefix and group depends on the
+// block size and the position alone.  Waits are bounded as in the other tensor-core kernels.
+#include <cuda.h>
+
+#include <algorithm>
+#include <vector>
+
+#include "js_common.cuh"
+#include "js_model.h"
+#include "made_driver.cuh"
+#include "tc_common.cuh"
+
+namespace {
+
+constexpr int BM = TC_BM, BK = TC_BK;
+constexpr int NTH = 192;
+constexpr int NUP = 32;                      // most units of one layer inside a group
+constexpr int GMAX = 16;                     // most positions per group
+constexpr int A_BYTES = BM * BK * 2;
+constexpr int W_BYTES = NUP * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + W_BYTES;          // 20 KB, a multiple of 1 KB
+constexpr int MAX_STAGES = 6;
+constexpr int SMEM_DYN_MAX = 227 * 1024 - 4 * 1024;
+
+struct SwShared {
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tfull, tempty, gdone;
+    uint32_t tmem_base;
+    int stop;
+    float lut_s[2];
+    // geometry of the current group, per GEMM l (activations a[l] -> a[l+1])
+    int kin0[JS_MAXL + 1], nin[JS_MAXL + 1], u0[JS_MAXL + 1], nu[JS_MAXL + 1], kb_n[JS_MAXL + 1];
+    int cs[JS_MAXL + 1][GMAX + 2];           // cs[l][i] = units of a[l] with degree <= t0 + i   (l >= 1)
+    float bias_s[JS_MAXL + 1][NUP];
+};
+
+struct Geo { int kin0, kb_n, nin, u0, nu, npad; };
+
+struct SweepEngine {
+    const MadeDev &m;
+    const SweepDev &sw;
+    const RunArgs &r;
+    SwShared &sh;
+    uint8_t *ring;
+    float *V;            // [L+1][NUP][128]: prefix sums, then activations, of the group's units
+    float *X;            // [NUP][128]: encodings of the group's positions
+    float *Wg;           // [L+1][NUP][NUP]: weights between the group's units
+    float *Nz;           // [GMAX][128]: the group's noise
+    int warp, lane;
+    int stage = 0;
+    uint32_t spar = 0;
+    uint32_t tf_par = 0, te_par = 0, gd_par = 0;
+    bool dead = false;
+    uint32_t tmem_base = 0;
+    unsigned long long mma_flops = 0;
+
+    __device__ SweepEngine(const MadeDev &m_, const SweepDev &sw_, const RunArgs &r_, SwShared &sh_, uint8_t *ring_)
+        : m(m_), sw(sw_), r(r_), sh(sh_), ring(ring_)
+    {
+        warp = threadIdx.x >> 5;
+        lane = threadIdx.x & 31;
+        uint8_t *p = ring + (size_t)sw.n_stages * STAGE_BYTES;
+        V = reinterpret_cast<float *>(p);
+        p += (size_t)(m.L + 1) * NUP * BM * 4;
+        X = reinterpret_cast<float *>(p);
+        p += (size_t)NUP * BM * 4;
+        Wg = reinterpret_cast<float *>(p);
+        p += (size_t)(m.L + 1) * NUP * NUP * 4;
+        Nz = reinterpret_cast<float *>(p);
+    }
+
+    // units of a[l] with degree <= d (a[0]: the positions themselves, degree = position + 1)
+    __device__ int cnt(int l, int d) const { return l == 0 ? d : __ldg(&sw.cnt[l][d]); }
+
+    // group [t0, t1) of a block ending at b: hidden degrees (t0, hi] are evaluated inside it
+    __device__ Geo geo(int l, int t0, int t1, int hi) const
+    {
+        Geo g;
+        g.kin0 = cnt(l, t0);
+        g.kb_n = (g.kin0 + BK - 1) / BK;
+        g.nin = cnt(l, hi) - g.kin0;
+        if (l < m.L) {
+            g.u0 = cnt(l + 1, t0);
+            g.nu = cnt(l + 1, hi) - g.u0;
+        } else {
+            g.u0 = t0;
+            g.nu = t1 - t0;
+        }
+        g.npad = (g.nu + 15) & ~15;
+        return g;
+    }
+
+    __device__ uint8_t *stage_a(int s) const { return ring + (size_t)s * STAGE_BYTES; }
+    __device__ uint8_t *stage_b(int s) const { return ring + (size_t)s * STAGE_BYTES + A_BYTES; }
+    __device__ uint32_t stage_parity() const { return (spar >> stage) & 1u; }
+    __device__ void advance_stage()
+    {
+        spar ^= 1u << stage;
+        if (++stage == sw.n_stages) stage = 0;
+    }
+
+    // ------------------------------------------------------------------ roles
+    __device__ void producer(int rt, int slot, int a, int b)
+    {
+        int kb_old[JS_MAXL + 1];
+        for (int l = 0; l <= m.L; ++l) kb_old[l] = cnt(l, a) / BK;
+        for (int t0 = a; t0 < b && !dead; t0 += sw.G) {
+            const int t1 = min(t0 + sw.G, b), hi = min(t1, b - 1);
+            // the previous group's activations (or the job's start values) are in F
+            if (!mbar_wait(&sh.gdone, gd_par, r.ctl)) { dead = true; break; }
+            gd_par ^= 1u;
+            fence_proxy_async();
+            for (int l = 0; l <= m.L && !dead; ++l) {
+                const Geo g = geo(l, t0, t1, hi);
+                if (g.nu == 0) continue;
+                const uint32_t bytes = A_BYTES + (uint32_t)g.npad * BK * 2;
+                mma_flops += 2ull * BM * BK * (unsigned long long)g.npad * (unsigned long long)g.kb_n;
+                for (int kb = 0; kb < g.kb_n; ++kb) {
+                    if (!mbar_wait(&sh.empty[stage], stage_parity() ^ 1u, r.ctl)) { dead = true; break; }
+                    mbar_expect_tx(&sh.full[stage], bytes);
+                    if (kb < kb_old[l])
+                        tma_load_2d(smem_u32(stage_a(stage)), sw.tmAold + l, &sh.full[stage], kb * BK, rt * BM);
+                    else
+                        tma_load_3d(smem_u32(stage_a(stage)), sw.tmF + l, &sh.full[stage], (kb - kb_old[l]) * BK, 0, slot);
+                    for (int i = 0; i < g.npad / 16; ++i)
+                        tma_load_2d(smem_u32(stage_b(stage)) + i * 16 * BK * 2, sw.tmW16 + l, &sh.full[stage], kb * BK,
+                                    g.u0 + i * 16);
+                    advance_stage();
+                }
+            }
+        }
+    }
+
+    __device__ void mma_issuer(int a, int b)
+    {
+        for (int t0 = a; t0 < b && !dead; t0 += sw.G) {
+            const int t1 = min(t0 + sw.G, b), hi = min(t1, b - 1);
+            // the epilogue has read the previous group's accumulators
+            if (!mbar_wait(&sh.tempty, te_par ^ 1u, r.ctl)) { dead = true; break; }
+            te_par ^= 1u;
+            tc_fence_after();
+            bool any = false;
+            for (int l = 0; l <= m.L && !dead; ++l) {
+                const Geo g = geo(l, t0, t1, hi);
+                if (g.nu == 0) continue;
+                const uint32_t idesc = instr_desc_bf16(g.npad);
+                const uint32_t d_tmem = tmem_base + (uint32_t)(l * NUP);
+                for (int kb = 0; kb < g.kb_n; ++kb) {
+                    if (!mbar_wait(&sh.full[stage], stage_parity(), r.ctl)) { dead = true; break; }
+                    tc_fence_after();
+                    const uint64_t adesc = smem_desc_sw128(smem_u32(stage_a(stage)));
+                    const uint64_t bdesc = smem_desc_sw128(smem_u32(stage_b(stage)));
+#pragma unroll
+                    for (int k = 0; k < BK / 16; ++k)
+                        umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
+                                  (kb > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(&sh.empty[stage]);
+                    advance_stage();
+                    any = true;
+                }
+            }
+            if (dead) break;
+            if (any) umma_commit(&sh.tfull);
+            else mbar_arrive(&sh.tfull);          // a group with empty prefixes (the very first positions)
+        }
+    }
+
+    __device__ void ep_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+    // start of a job: the job's buffer F holds, per layer, the units from the K block that contains
+    // the block's first old unit onwards: copies of the old activations up to degree a, zeros after
+    __device__ void job_init(int rt, int slot, int a, int b)
+    {
+        const int row = (warp & 3) * 32 + lane;
+        const size_t esz = 2;
+        for (int l = 0; l <= m.L; ++l) {
+            const int k_old = cnt(l, a), kb0 = (k_old / BK) * BK;
+            const int ncopy = k_old - kb0;
+            const int cols = min(sw.WF[l], ((cnt(l, min(b, m.T)) - kb0 + BK - 1) / BK) * BK);
+            __nv_bfloat16 *f = sw.F[l] + ((size_t)slot * BM + row) * sw.WF[l];
+            const __nv_bfloat16 *old = (const __nv_bfloat16 *)m.a[l] + (size_t)(rt * BM + row) * m.n[l] + kb0;
+            for (int c = 0; c < cols; c += 8) {
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (c + 8 <= ncopy) {
+                    v = __ldcg(reinterpret_cast<const uint4 *>(old + c));
+                } else if (c < ncopy) {
+                    __nv_bfloat16 tmp[8];
+                    for (int i = 0; i < 8; ++i) tmp[i] = c + i < ncopy ? old[c + i] : __float2bfloat16_rn(0.0f);
+                    v = *reinterpret_cast<const uint4 *>(tmp);
+                }
+                *reinterpret_cast<uint4 *>(f + c) = v;
+            }
+            (void)esz;
+        }
+        fence_proxy_async();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh.gdone);
+    }
+
+    __device__ void epilogue(int rt, int slot, int a, int b, bool &row_changed)
+    {
+        const int q = warp & 3, row = q * 32 + lane, tid = threadIdx.x - 64;
+        const int smp = rt * BM + row;
+        const bool valid = smp < r.batch;
+        const int L = m.L;
+        int kb_old[JS_MAXL + 1];
+        for (int l = 0; l <= L; ++l) kb_old[l] = cnt(l, a) / BK;
+        job_init(rt, slot, a, b);
+        for (int t0 = a; t0 < b && !dead; t0 += sw.G) {
+            const int t1 = min(t0 + sw.G, b), hi = min(t1, b - 1), ng = t1 - t0;
+            // ---- geometry, small tables, the weights between the group's units, noise (while the GEMMs run)
+            ep_sync();                                   // everybody is done with the previous group's tables
+            if (tid <= L) {
+                const Geo g = geo(tid, t0, t1, hi);
+                sh.kin0[tid] = g.kin0; sh.nin[tid] = g.nin; sh.u0[tid] = g.u0; sh.nu[tid] = g.nu; sh.kb_n[tid] = g.kb_n;
+            }
+            for (int i = tid; i < (L + 1) * (GMAX + 2); i += 128) {
+                const int l = i / (GMAX + 2), k = i % (GMAX + 2);
+                if (l >= 1) sh.cs[l][k] = cnt(l, min(t0 + k, m.T));
+            }
+            ep_sync();
+            for (int l = 0; l <= L; ++l) {
+                const int nu = sh.nu[l], nin = sh.nin[l], u0 = sh.u0[l], kin0 = sh.kin0[l];
+                const __nv_bfloat16 *Wl = (const __nv_bfloat16 *)m.W[l];
+                const int K = m.n[l];
+                for (int i = tid; i < NUP * NUP; i += 128) {
+                    const int j = i / NUP, k = i % NUP;
+                    float w = 0.0f;
+                    if (j < nu && k < nin) w = __bfloat162float(Wl[(size_t)(u0 + j) * K + kin0 + k]);
+                    Wg[(l * NUP + j) * NUP + k] = w;
+                }
+                if (tid < NUP) sh.bias_s[l][tid] = tid < nu ? m.bias[l][u0 + tid] : 0.0f;
+            }
+            for (int i = 0; i < GMAX; ++i) Nz[i * BM + row] = (valid && i < ng) ? r.noise[(size_t)smp * m.T + t0 + i] : 0.0f;
+            for (int k = 0; k < NUP; ++k) X[k * BM + row] = 0.0f;
+            ep_sync();
+            // ---- prefix sums out of tensor memory
+            if (!mbar_wait(&sh.tfull, tf_par, r.ctl)) { dead = true; break; }
+            tf_par ^= 1u;
+            tc_fence_after();
+            for (int l = 0; l <= L; ++l) {
+                float v[32];
+                if (sh.nu[l] > 0 && sh.kb_n[l] > 0) {
+                    tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(l * NUP), v);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = 0.0f;
+                }
+#pragma unroll
+                for (int i = 0; i < 32; ++i) V[(l * NUP + i) * BM + row] = v[i];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh.tempty);
+            // ---- the group's positions in order, thread = sample row
+            for (int i = 0; i < ng; ++i) {
+                const int t = t0 + i;
+                float z = V[(L * NUP + i) * BM + row] + sh.bias_s[L][i];
+                {
+                    const float *wrow = Wg + (L * NUP + i) * NUP;
+                    const int nin = sh.nin[L];
+                    for (int k = 0; k < nin; ++k) z = fmaf(wrow[k], V[((L - 1) * NUP + k) * BM + row], z);
+                }
+                const int xn = js_sample_binary(r.nk, z, Nz[i * BM + row]);
+                if (valid) {
+                    uint8_t *xp = r.x + (size_t)smp * m.T + t;
+                    if (*xp != (uint8_t)xn) { *xp = (uint8_t)xn; row_changed = true; }
+                }
+                X[i * BM + row] = sh.lut_s[xn];
+                if (t + 1 > hi) continue;
+                // the hidden units that position t makes computable: degree t + 1
+                for (int l = 0; l < L; ++l) {
+                    const int j0 = sh.cs[l + 1][i] - sh.u0[l], j1 = sh.cs[l + 1][i + 1] - sh.u0[l];
+                    const int nin = sh.nin[l];
+                    const float *in = l == 0 ? X : V + (size_t)(l - 1) * NUP * BM;
+                    for (int j = j0; j < j1; ++j) {
+                        float pre = V[(l * NUP + j) * BM + row] + sh.bias_s[l][j];
+                        const float *wrow = Wg + (l * NUP + j) * NUP;
+                        for (int k = 0; k < nin; ++k) pre = fmaf(wrow[k], in[k * BM + row], pre);
+                        V[(l * NUP + j) * BM + row] = __bfloat162float(__float2bfloat16_rn(tc_act_fn(m.act, pre)));
+                    }
+                }
+            }
+            // ---- the group's activations into F, for the GEMMs of the groups that follow
+            if (t1 < b) {
+                {
+                    __nv_bfloat16 *f = sw.F[0] + ((size_t)slot * BM + row) * sw.WF[0] + (t0 - kb_old[0] * BK);
+                    for (int i = 0; i < ng; ++i) f[i] = __float2bfloat16_rn(X[i * BM + row]);
+                }
+                for (int l = 1; l <= L; ++l) {
+                    const int n = sh.nin[l];
+                    __nv_bfloat16 *f = sw.F[l] + ((size_t)slot * BM + row) * sw.WF[l] + (sh.kin0[l] - kb_old[l] * BK);
+                    for (int j = 0; j < n; ++j) f[j] = __float2bfloat16_rn(V[((l - 1) * NUP + j) * BM + row]);
+                }
+                fence_proxy_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sh.gdone);
+            }
+        }
+    }
+};
+
+__global__ void __launch_bounds__(NTH, 1)
+made_sweep_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ SweepDev sw, const __grid_constant__ RunArgs r)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ SwShared sh;
+    uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
+        mbar_init(&sh.tfull, 1);
+        mbar_init(&sh.tempty, 4);
+        mbar_init(&sh.gdone, 4);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_proxy_async();
+        sh.lut_s[0] = m.lut[0];
+        sh.lut_s[1] = m.lut[1];
+    }
+    if (warp == 1) tmem_alloc(&sh.tmem_base, 512);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+
+    SweepEngine e(m, sw, r, sh, ring);
+    e.tmem_base = sh.tmem_base;
+    // jobs: (row tile, block), the blocks with the longest prefixes first
+    const int B = r.block, nblk = (m.T + B - 1) / B, MT = (r.batch + BM - 1) / BM;
+    const int njobs = MT * (nblk - r.blk_lo);
+    for (int job = blockIdx.x; job < njobs; job += gridDim.x) {
+        const int blk = nblk - 1 - job / MT, rt = job % MT;
+        const int a = blk * B, b = min(a + B, m.T);
+        // The accumulators and the ring are idle between jobs; the roles meet here so that a job's
+        // start values are never written while the previous job is still being read, and so that
+        // all of them see the same answer to "has a wait given up".
+        __syncthreads();
+        if (threadIdx.x == 0) sh.stop = ld_volatile_i32(&r.ctl->abort);
+        __syncthreads();
+        if (sh.stop) break;
+        if (warp == 0) {
+            if (e.lane == 0) e.producer(rt, blockIdx.x, a, b);
+        } else if (warp == 1) {
+            if (e.lane == 0) e.mma_issuer(a, b);
+        } else {
+            bool row_changed = false;
+            e.epilogue(rt, blockIdx.x, a, b, row_changed);
+            const int smp = rt * BM + (warp & 3) * 32 + e.lane;
+            if (row_changed && smp < r.batch) r.smp_changed[smp] = 1;
+        }
+        __syncwarp();
+    }
+    DriverResult res = {JS_OK, 0, m.T, !e.dead};
+    tc_fence_before();
+    __syncthreads();
+    if (!res.alive || ld_volatile_i32(&r.ctl->abort) != 0) {
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);      // let copies still in flight land
+        res.alive = false;
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(e.tmem_base, 512);
+    }
+    driver_finish(r, res, 0, 0, e.mma_flops, 0);
+}
+
+// Per-sample bookkeeping of Jacobi-GS after outer iteration k (one CTA): a sample whose iterate did
+// not change stops counting; the flags are cleared for the next iteration and the host learns
+// whether anything changed.
+__global__ void jgs_book_kernel(int batch, int k, int at_cap, int *changed, int *done, int32_t *out_iters, int *any_out)
+{
+    __shared__ int any;
+    if (threadIdx.x == 0) any = 0;
+    __syncthreads();
+    for (int b = threadIdx.x; b < batch; b += blockDim.x) {
+        const int c = changed[b];
+        if (c) any = 1;
+        if (!done[b] && (c == 0 || at_cap)) {
+            done[b] = 1;
+            if (out_iters) out_iters[b] = k;
+        }
+        changed[b] = 0;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        *any_out = any;
+        __threadfence_system();
+    }
+}
+
+}  // namespace
+
+// --------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn sweep_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void *p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess)
+        return nullptr;
+    fn = (EncodeTiledFn)p;
+    return fn;
+}
+
+static bool sweep_encode(CUtensorMap *out, const void *base, int rank, const cuuint64_t *dims, const cuuint64_t *strides,
+                         const cuuint32_t *box)
+{
+    EncodeTiledFn fn = sweep_encode_fn();
+    if (!fn) return false;
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Builds what the sweeps need beside the tensor-core view of the model: prefix counts per degree,
+// the group size, the jobs' buffers F and the tensor maps.  Returns 1 if the model qualifies
+// (binary positions, sorted degrees, bf16), 0 if not, negative on CUDA errors.  Called on first use.
+int js_sweep_prepare(js_model *mo)
+{
+    if (mo->sweep_state != 0) return mo->sweep_state > 0 ? 1 : 0;
+    mo->sweep_state = -1;
+    const MadeDev &v = mo->made;
+    SweepDev &s = mo->sweep;
+    if (!mo->tc_ok || v.C != 1 || v.prec != JS_BF16 || !sweep_encode_fn()) return 0;
+    const int L = v.L, T = v.T;
+    // prefix counts; the group size is the largest one that keeps every layer's units of a group within NUP
+    std::vector<std::vector<int>> cnt(L + 1);
+    for (int l = 1; l <= L; ++l) {
+        cnt[l].assign(T + 1, 0);
+        const std::vector<int> &dg = mo->host_deg[l];
+        for (size_t i = 1; i < dg.size(); ++i)
+            if (dg[i] < dg[i - 1]) return 0;                       // needs sorted degrees
+        size_t p = 0;
+        for (int d = 0; d <= T; ++d) {
+            while (p < dg.size() && dg[p] <= d) ++p;
+            cnt[l][d] = (int)p;
+        }
+    }
+    int G = GMAX;
+    for (; G >= 1; G >>= 1) {
+        bool ok = true;
+        for (int l = 1; l <= L && ok; ++l)
+            for (int d = 0; d + G <= T && ok; ++d)
+                if (cnt[l][d + G] - cnt[l][d] > NUP) ok = false;
+        if (ok) break;
+    }
+    if (G < 1) return 0;
+    s.G = G;
+    const int fixed = (L + 1) * NUP * BM * 4 + NUP * BM * 4 + (L + 1) * NUP * NUP * 4 + GMAX * BM * 4;
+    s.n_stages = std::min(MAX_STAGES, (SMEM_DYN_MAX - 1024 - fixed) / STAGE_BYTES);
+    if (s.n_stages < 2) return 0;
+    s.smem_bytes = 1024 + s.n_stages * STAGE_BYTES + fixed;
+    int dev = 0, sms = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (sms < 1) return 0;
+    s.slots = sms;
+    auto fail = [&]() { cudaGetLastError(); return JS_ERR_CUDA; };
+    std::vector<CUtensorMap> mapsF(L + 1), mapsW(L + 1);
+    for (int l = 0; l <= L; ++l) {
+        if (l >= 1) {
+            void *p = nullptr;
+            if (cudaMalloc(&p, (T + 1) * sizeof(int)) != cudaSuccess) return fail();
+            mo->allocs.push_back(p);
+            if (cudaMemcpy(p, cnt[l].data(), (T + 1) * sizeof(int), cudaMemcpyHostToDevice) != cudaSuccess) return fail();
+            s.cnt[l] = (const int *)p;
+        } else {
+            s.cnt[l] = nullptr;
+        }
+        s.WF[l] = (v.n[l] + BK - 1) / BK * BK + BK;
+        void *f = nullptr;
+        const size_t bytes = (size_t)s.slots * BM * s.WF[l] * 2;
+        if (cudaMalloc(&f, bytes) != cudaSuccess) return fail();
+        mo->allocs.push_back(f);
+        if (cudaMemset(f, 0, bytes) != cudaSuccess) return fail();
+        s.F[l] = (__nv_bfloat16 *)f;
+        {
+            const cuuint64_t dims[3] = {(cuuint64_t)s.WF[l], (cuuint64_t)BM, (cuuint64_t)s.slots};
+            const cuuint64_t strides[2] = {(cuuint64_t)s.WF[l] * 2, (cuuint64_t)s.WF[l] * 2 * BM};
+            const cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BM, 1};
+            if (!sweep_encode(&mapsF[l], f, 3, dims, strides, box)) return 0;
+        }
+        {
+            const cuuint64_t dims[2] = {(cuuint64_t)v.n[l], (cuuint64_t)v.n[l + 1]};
+            const cuuint64_t strides[1] = {(cuuint64_t)v.n[l] * 2};
+            const cuuint32_t box[2] = {(cuuint32_t)BK, 16};
+            if (!sweep_encode(&mapsW[l], v.W[l], 2, dims, strides, box)) return 0;
+        }
+    }
+    void *pf = nullptr, *pw = nullptr;
+    if (cudaMalloc(&pf, (L + 1) * sizeof(CUtensorMap)) != cudaSuccess) return fail();
+    mo->allocs.push_back(pf);
+    if (cudaMalloc(&pw, (L + 1) * sizeof(CUtensorMap)) != cudaSuccess) return fail();
+    mo->allocs.push_back(pw);
+    if (cudaMemcpy(pf, mapsF.data(), (L + 1) * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess) return fail();
+    if (cudaMemcpy(pw, mapsW.data(), (L + 1) * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess) return fail();
+    s.tmF = (const CUtensorMap *)pf;
+    s.tmW16 = (const CUtensorMap *)pw;
+    s.tmAold = mo->tc.tmA;
+    {
+        void *p = nullptr;
+        if (cudaMalloc(&p, 2 * (size_t)mo->rows * sizeof(int)) != cudaSuccess) return fail();
+        mo->allocs.push_back(p);
+        if (cudaMemset(p, 0, 2 * (size_t)mo->rows * sizeof(int)) != cudaSuccess) return fail();
+        mo->sw_flags = (int *)p;
+        if (cudaHostAlloc((void **)&mo->h_any, sizeof(int), cudaHostAllocMapped) != cudaSuccess) return fail();
+        if (cudaHostGetDevicePointer((void **)&mo->d_any, mo->h_any, 0) != cudaSuccess) return fail();
+    }
+    if (cudaFuncSetAttribute(made_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_MAX) != cudaSuccess) {
+        cudaGetLastError();
+        return 0;
+    }
+    mo->sweep_state = 1;
+    return 1;
+}
+
+// One launch: sweeps of every block >= r.blk_lo (block size r.block) for every row tile.
+int js_launch_made_sweep(const js_model *mo, const RunArgs &r, cudaStream_t stream)
+{
+    const SweepDev &s = mo->sweep;
+    const int nblk = (mo->made.T + r.block - 1) / r.block, MT = (r.batch + BM - 1) / BM;
+    const int njobs = MT * (nblk - r.blk_lo);
+    if (njobs < 1) return (int)cudaErrorInvalidValue;
+    const int grid = std::min(njobs, s.slots);
+    made_sweep_kernel<<<grid, NTH, s.smem_bytes, stream>>>(mo->made, s, r);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? 0 : (int)e;
+}
+
+int js_launch_jgs_book(const js_model *mo, int batch, int k, int at_cap, int32_t *out_iters, cudaStream_t stream)
+{
+    jgs_book_kernel<<<1, 256, 0, stream>>>(batch, k, at_cap, mo->sw_flags, mo->sw_flags + mo->rows, out_iters, mo->d_any);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? 0 : (int)e;
+}

@@ -67,7 +67,7 @@ struct TcEngine {
     uint8_t *staging;
     const int *meta;               // tile metadata in shared memory: per layer kb_end[nt], dmin[nt], dmax[nt]
     unsigned epoch = 0;
-    unsigned long long issued = 0, skipped = 0;
+    unsigned long long issued = 0, skipped = 0, mma_flops = 0, weight_bytes = 0;
     int warp, lane;
     // pipeline state, advanced identically by the roles that share it
     int stage = 0;
@@ -332,6 +332,8 @@ struct TcEngine {
         Unit u;
         while (!dead && next_unit(l, e, e_end, nt_lo, nt_hi, MT, u)) {
             issued++;
+            mma_flops += 2ull * BM * BK * (unsigned long long)ly.bn * (unsigned long long)(u.kb1 - u.kb0);
+            if (u.mt == 0) weight_bytes += 2ull * BK * (unsigned long long)ly.bn * (unsigned long long)(u.kb1 - u.kb0);
             for (int kb = u.kb0; kb < u.kb1; ++kb) {
                 if (!mbar_wait(&sh.empty[stage], stage_parity() ^ 1u, r.ctl)) { dead = true; break; }
                 mbar_expect_tx(&sh.full[stage], bytes);
@@ -1051,7 +1053,7 @@ made_tc_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ TcDev 
         tc_fence_after();
         tmem_dealloc(e.tmem_base, 512);
     }
-    driver_finish(r, res, e.issued, e.skipped);
+    driver_finish(r, res, e.issued, e.skipped, e.mma_flops, e.weight_bytes);
 }
 
 }  // namespace

@@ -11,10 +11,11 @@ not itself a near-tie.  Excused samples and positions are counted and returned.
 MARGIN is 1e-3.  A deep bf16 network needs more: every hidden value is rounded to 8
 mantissa bits, the oracle rounds double sums and the kernel fp32 sums, so now and then a
 hidden unit rounds the other way and moves a logit by about one bf16 step of an
-activation times a weight.  For such a model the caller measures E, the largest absolute
-difference between the two sides' teacher-forced logits (which must itself pass the
-relative logit tolerance), and passes margin = max(1e-3, 2 E): two logits that may each
-be off by E can swap order when they are closer than 2 E.
+activation times a weight.  For such a model the caller derives a bound E on the logit
+difference from the model alone (bf16 spacing of the largest activation times the largest
+weight of the last layer), asserts the measured difference against it, and passes
+margin = 2 E: two logits that may each be off by E can swap order when they are closer
+than 2 E.  Such a model does not meet the plain rule, and its test says so.
 """
 from __future__ import annotations
 

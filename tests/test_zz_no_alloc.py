@@ -77,3 +77,22 @@ def test_noalloc_rejects_shapes_beyond_its_scratch():
     with pytest.raises(p.JsError) as e:
         p.jacobi_sample_noalloc(cfg.D, cfg.C, cfg.H, cfg.act, W, b, lut, noise, cfg.noise_kind, None, 0, out, None)
     assert e.value.code == p.JS_ERR_ARG and "scratch" in str(e.value)
+
+
+def test_noalloc_row_without_a_finite_score_gets_class_zero():
+    """Weights or noise from the caller may hold NaN: a position whose scores are all NaN has no
+    largest one.  The call must come back cleanly with class 0 there, like jacobi_sample."""
+    p = _pkg()
+    cfg = CASES[2]
+    W, b = si.made_weights(cfg)
+    bad = 3
+    b[-1][bad * cfg.C:(bad + 1) * cfg.C] = np.nan
+    dW = [torch.from_numpy(w).cuda() for w in W]
+    db = [torch.from_numpy(v).cuda() for v in b]
+    dlut = torch.from_numpy(si.made_lut(cfg)).cuda()
+    noise = torch.from_numpy(si.draw_noise(cfg)).cuda()
+    got = torch.full((cfg.batch, cfg.D), 255, dtype=torch.uint8, device="cuda")
+    rc = p.jacobi_sample_noalloc(cfg.D, cfg.C, cfg.H, cfg.act, dW, db, dlut, noise, cfg.noise_kind, None, 0, got, None)
+    assert rc == 0
+    x = got.cpu().numpy()
+    assert np.all(x[:, bad] == 0) and x.max() < cfg.C
