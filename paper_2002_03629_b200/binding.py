@@ -10,7 +10,7 @@ import numpy as np
 import torch
 
 JS_JACOBI, JS_GAUSS_SEIDEL, JS_GS_JACOBI, JS_JACOBI_GS = 0, 1, 2, 3
-JS_NOISE_UNIFORM_ICDF, JS_NOISE_LOGISTIC, JS_NOISE_GUMBEL = 0, 1, 2
+JS_NOISE_UNIFORM_ICDF, JS_NOISE_LOGISTIC, JS_NOISE_GUMBEL, JS_NOISE_UNIFORM_CAT = 0, 1, 2, 3
 JS_ACT_RELU, JS_ACT_GELU_TANH = 0, 1
 JS_F32, JS_BF16 = 0, 1
 JS_OK, JS_NOT_CONVERGED = 0, 1

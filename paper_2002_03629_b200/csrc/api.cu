@@ -180,7 +180,7 @@ int common_scratch(js_model *m, int T)
 bool noise_kind_ok(const js_model *m, int nk)
 {
     const int C = m->kind == 0 ? m->made.C : m->conv_C;
-    if (nk == JS_NOISE_GUMBEL) return C > 1;
+    if (nk == JS_NOISE_GUMBEL || nk == JS_NOISE_UNIFORM_CAT) return C > 1;
     if (nk == JS_NOISE_UNIFORM_ICDF || nk == JS_NOISE_LOGISTIC) return C == 1;
     return false;
 }
@@ -341,6 +341,7 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
 {
     const MadeDev &v = m->made;
     if (m->kind == 1 && r.kmode == KM_JACOBI_GS) return JS_ERR_UNSUPPORTED;
+    if (m->kind == 1 && r.nk == JS_NOISE_UNIFORM_CAT && r.kmode != KM_FORWARD) return JS_ERR_UNSUPPORTED;
     // the sweeps: the strict order with cached hidden units, and Algorithm 2
     if (r.kmode == KM_SEQ && m->opt_seq_skip == 2 && sweeps_usable(m, r)) return run_sweep_sequential(m, r, st);
     if (r.kmode == KM_JACOBI_GS && sweeps_usable(m, r)) return run_jacobi_gs_tc(m, r, st);
@@ -529,7 +530,8 @@ int jacobi_sample_host(const js_model *cm, int batch, const float *noise_host, i
         HOST_TRY(cudaEventRecord(m->ev_copy, cs));
         HOST_TRY(cudaStreamWaitEvent(st, m->ev_copy, 0));       // the start iterate is needed at once
     }
-    HOST_TRY(cudaMemcpyAsync(m->st_noise, noise_host, (size_t)batch * T * C * sizeof(float), cudaMemcpyHostToDevice, cs));
+    HOST_TRY(cudaMemcpyAsync(m->st_noise, noise_host, (size_t)batch * T * (nk == JS_NOISE_GUMBEL ? C : 1) * sizeof(float),
+                             cudaMemcpyHostToDevice, cs));
     // copies of one stream run in order: this word changes after the noise has arrived
     *m->h_nflag = ++m->n_uploads;
     HOST_TRY(cudaMemcpyAsync(m->d_nflag, m->h_nflag, sizeof(unsigned), cudaMemcpyHostToDevice, cs));

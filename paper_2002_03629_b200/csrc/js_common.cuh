@@ -4,6 +4,7 @@
 
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
+#include <limits.h>
 #include <stdint.h>
 
 #include "../../include/jacobi_sample.h"
@@ -135,6 +136,64 @@ __device__ __forceinline__ int js_sample_binary(int nk, float z, float noise)
         return noise < p ? 1 : 0;
     }
     return (z + noise) > 0.0f ? 1 : 0;
+}
+
+// x_t of a C-way position, computed by one warp from the position's logits (Appendix A.3).
+//   JS_NOISE_GUMBEL       noise = C Gumbel numbers: argmax_c (z_c + g_c), lowest index among equals
+//   JS_NOISE_UNIFORM_CAT  noise = one uniform number u: the first class c with u * S < sum_{i<=c} e_i,
+//                         e_i = exp(z_i - max z), S = sum of all e_i (inverse CDF of the softmax)
+// Every lane returns the class; a row without a finite score gives class 0.
+__device__ __forceinline__ int js_warp_sample_cat(int nk, const float *zz, const float *noise, int C, int lane)
+{
+    if (nk == JS_NOISE_UNIFORM_CAT) {
+        float mx = -INFINITY;
+        for (int c = lane; c < C; c += 32) mx = fmaxf(mx, zz[c]);
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        // two passes over the classes in chunks of 32 (lane = class inside the chunk): the total,
+        // then the running sums; a chunk's running sums are an inclusive scan across the lanes
+        float total = 0.0f;
+        for (int c0 = 0; c0 < C; c0 += 32) {
+            float e = (c0 + lane < C) ? expf(zz[c0 + lane] - mx) : 0.0f;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const float o = __shfl_up_sync(0xffffffffu, e, off);
+                if (lane >= off) e += o;
+            }
+            total += __shfl_sync(0xffffffffu, e, 31);
+        }
+        const float target = noise[0] * total;
+        float carry = 0.0f;
+        int found = INT_MAX;
+        for (int c0 = 0; c0 < C && found == INT_MAX; c0 += 32) {
+            float e = (c0 + lane < C) ? expf(zz[c0 + lane] - mx) : 0.0f;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const float o = __shfl_up_sync(0xffffffffu, e, off);
+                if (lane >= off) e += o;
+            }
+            const float run = carry + e;
+            const unsigned hit = __ballot_sync(0xffffffffu, c0 + lane < C && target < run);
+            if (hit) found = c0 + __ffs((int)hit) - 1;
+            carry += __shfl_sync(0xffffffffu, e, 31);
+        }
+        if (found == INT_MAX) found = (total == total) ? C - 1 : 0;      // u at the very top, or no finite score
+        return found;
+    }
+    float best = -INFINITY;
+    int bi = INT_MAX;
+    for (int c = lane; c < C; c += 32) {
+        const float v = zz[c] + noise[c];
+        if (v > best) { best = v; bi = c; }
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        const float ov = __shfl_xor_sync(0xffffffffu, best, off);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
+        if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+    }
+    if ((unsigned)bi >= (unsigned)C) bi = 0;      // no finite score in the row: class 0
+    return bi;
 }
 
 template <typename T> __device__ __forceinline__ float to_f32(T v);

@@ -158,21 +158,7 @@ __device__ void sample_phase(const MadeDev &m, const RunArgs &r, const float *z,
     for (size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; i < n; i += warps) {
         const int b = (int)(i / np), d = plo + (int)(i % np);
         const size_t at = (size_t)b * T_ + d;
-        const float *zz = z + at * C;
-        const float *gg = r.noise + at * C;
-        float best = -INFINITY;
-        int bi = INT_MAX;
-        for (int c = lane; c < C; c += 32) {
-            const float v = zz[c] + gg[c];
-            if (v > best) { best = v; bi = c; }
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, best, off);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-            if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
-        }
-        if ((unsigned)bi >= (unsigned)C) bi = 0;      // no finite score in the row: class 0
+        const int bi = js_warp_sample_cat(r.nk, z + at * C, r.noise + (r.nk == JS_NOISE_GUMBEL ? at * C : at), C, lane);
         if (lane == 0 && bi != r.x[at]) {
             r.x[at] = (uint8_t)bi;
             a0[at] = from_f32<T>(m.lut[bi]);
@@ -304,21 +290,7 @@ __device__ void jgs_commit_phase(const MadeDev &m, const RunArgs &r, int j, int 
         const int t = (blk_lo + (int)(it / r.batch)) * B + j;
         if (t >= m.T) continue;
         const size_t at = (size_t)b * m.T + t;
-        const float *zz = m.logits + at * C;
-        const float *gg = r.noise + at * C;
-        float best = -INFINITY;
-        int bi = INT_MAX;
-        for (int c = lane; c < C; c += 32) {
-            const float v = zz[c] + gg[c];
-            if (v > best) { best = v; bi = c; }
-        }
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const float ov = __shfl_xor_sync(0xffffffffu, best, off);
-            const int oi = __shfl_xor_sync(0xffffffffu, bi, off);
-            if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
-        }
-        if ((unsigned)bi >= (unsigned)C) bi = 0;
+        const int bi = js_warp_sample_cat(r.nk, m.logits + at * C, r.noise + (r.nk == JS_NOISE_GUMBEL ? at * C : at), C, lane);
         if (lane == 0) {
             r.x[at] = (uint8_t)bi;
             ((T *)m.a[0])[at] = from_f32<T>(m.lut[bi]);

@@ -37,7 +37,7 @@ namespace {
 constexpr int BM = TC_BM, BK = TC_BK;
 constexpr int NTH = 192;
 constexpr int NUP = 32;                      // most units of one layer inside a group
-constexpr int GMAX = 16;                     // most positions per group
+constexpr int GMAX = 32;                     // most positions per group
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int W_BYTES = NUP * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + W_BYTES;          // 20 KB, a multiple of 1 KB
@@ -57,13 +57,34 @@ struct SwShared {
 
 struct Geo { int kin0, kb_n, nin, u0, nu, npad; };
 
+// shared-memory accesses by 32-bit shared address: the position loop runs on one warp per scheduler, and
+// a generic load (which is what a pointer kept in a structure compiles to) waits much longer than ld.shared
+__device__ __forceinline__ float4 lds_f4(uint32_t a)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts_f4(uint32_t a, float4 v)
+{
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(a), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
+}
+__device__ __forceinline__ float lds_f(uint32_t a)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ void sts_f(uint32_t a, float v) { asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory"); }
+
 struct SweepEngine {
     const MadeDev &m;
     const SweepDev &sw;
     const RunArgs &r;
     SwShared &sh;
     uint8_t *ring;
-    float *V;            // [L+1][NUP][128]: prefix sums, then activations, of the group's units
+    float *V;            // [L+1][128 rows][NUP]: running sums, then activations, of the group's units; a row's
+                         // eight 16-byte chunks are permuted by the row number (conflict-free 16-byte accesses)
     float *X;            // [NUP][128]: encodings of the group's positions
     float *Wg;           // [L+1][NUP][NUP]: weights between the group's units
     float *Nz;           // [GMAX][128]: the group's noise
@@ -88,6 +109,16 @@ struct SweepEngine {
         Wg = reinterpret_cast<float *>(p);
         p += (size_t)(m.L + 1) * NUP * NUP * 4;
         Nz = reinterpret_cast<float *>(p);
+    }
+
+    // optional device timeline (JS_OPT_TRACE, js_get_trace) of the first CTA: one row of stamps per group;
+    // slots: 0 operands may be loaded, 1 last MMA issued, 2 group tables ready, 3 prefix sums complete,
+    // 4 prefix sums read, 5 positions done, 6 activations stored
+    int group_no = 0;
+    __device__ void trace(int slot) const
+    {
+        if (r.trace == nullptr || blockIdx.x != 0 || group_no >= JS_TRACE_PHASES) return;
+        r.trace[(size_t)group_no * JS_TRACE_SLOTS + slot] = global_ns();
     }
 
     // units of a[l] with degree <= d (a[0]: the positions themselves, degree = position + 1)
@@ -131,6 +162,7 @@ struct SweepEngine {
             if (!mbar_wait(&sh.gdone, gd_par, r.ctl)) { dead = true; break; }
             gd_par ^= 1u;
             fence_proxy_async();
+            trace(0);
             for (int l = 0; l <= m.L && !dead; ++l) {
                 const Geo g = geo(l, t0, t1, hi);
                 if (g.nu == 0) continue;
@@ -149,6 +181,7 @@ struct SweepEngine {
                     advance_stage();
                 }
             }
+            group_no++;
         }
     }
 
@@ -183,10 +216,60 @@ struct SweepEngine {
             if (dead) break;
             if (any) umma_commit(&sh.tfull);
             else mbar_arrive(&sh.tfull);          // a group with empty prefixes (the very first positions)
+            trace(1);
+            group_no++;
         }
     }
 
     __device__ void ep_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+    // unit j of the group in layer slot l, sample row `row`: its shared-memory address
+    __device__ uint32_t vat(int l, int j, int row) const
+    {
+        return smem_u32(V) + 4u * (uint32_t)(((l * BM + row) * NUP) + ((((j >> 2) ^ (row & 7)) << 2) | (j & 3)));
+    }
+
+    // source k of a[l] has the value `val`: add its contribution to the running sums of the group's units
+    // of a[l+1] (masked weights are zero where the target may not read the source)
+    __device__ void scatter(int l, int k, float val, int row)
+    {
+        // the row's 32 running sums as eight 16-byte accesses, all loads before all stores: one warp per
+        // scheduler cannot hide the latency of a load that waits behind a store it might alias
+        const uint32_t w4 = smem_u32(Wg) + 4u * (uint32_t)((l * NUP + k) * NUP);
+        const uint32_t v4 = smem_u32(V) + 4u * (uint32_t)((l * BM + row) * NUP);
+        const int sw7 = row & 7;
+        float4 w[NUP / 4], x[NUP / 4];
+#pragma unroll
+        for (int c = 0; c < NUP / 4; ++c) w[c] = lds_f4(w4 + 16u * c);
+#pragma unroll
+        for (int c = 0; c < NUP / 4; ++c) x[c] = lds_f4(v4 + 16u * (uint32_t)(c ^ sw7));
+#pragma unroll
+        for (int c = 0; c < NUP / 4; ++c) {
+            x[c].x = fmaf(w[c].x, val, x[c].x);
+            x[c].y = fmaf(w[c].y, val, x[c].y);
+            x[c].z = fmaf(w[c].z, val, x[c].z);
+            x[c].w = fmaf(w[c].w, val, x[c].w);
+        }
+#pragma unroll
+        for (int c = 0; c < NUP / 4; ++c) sts_f4(v4 + 16u * (uint32_t)(c ^ sw7), x[c]);
+    }
+
+    // n consecutive values (unit j = 0..n-1 of layer slot l, or the group's encodings when l < 0) of this
+    // thread's row as bf16 to dst[0..n): single elements up to a 16-byte boundary, then eight at a time
+    __device__ float run_val(int l, int j, int row) const { return l < 0 ? X[j * BM + row] : lds_f(vat(l, j, row)); }
+    __device__ void store_run(__nv_bfloat16 *dst, int l, int row, int n)
+    {
+        int j = 0;
+        for (; j < n && (reinterpret_cast<uintptr_t>(dst + j) & 15u) != 0; ++j) dst[j] = __float2bfloat16_rn(run_val(l, j, row));
+        for (; j + 8 <= n; j += 8) {
+            float x[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) x[i] = run_val(l, j + i, row);
+            *reinterpret_cast<uint4 *>(dst + j) = make_uint4(pack_bf16x2(x[0], x[1]), pack_bf16x2(x[2], x[3]),
+                                                             pack_bf16x2(x[4], x[5]), pack_bf16x2(x[6], x[7]));
+        }
+        for (; j < n; ++j) dst[j] = __float2bfloat16_rn(run_val(l, j, row));
+    }
 
     // start of a job: the job's buffer F holds, per layer, the units from the K block that contains
     // the block's first old unit onwards: copies of the old activations up to degree a, zeros after
@@ -244,21 +327,48 @@ struct SweepEngine {
                 const int nu = sh.nu[l], nin = sh.nin[l], u0 = sh.u0[l], kin0 = sh.kin0[l];
                 const __nv_bfloat16 *Wl = (const __nv_bfloat16 *)m.W[l];
                 const int K = m.n[l];
-                for (int i = tid; i < NUP * NUP; i += 128) {
-                    const int j = i / NUP, k = i % NUP;
-                    float w = 0.0f;
-                    if (j < nu && k < nin) w = __bfloat162float(Wl[(size_t)(u0 + j) * K + kin0 + k]);
-                    Wg[(l * NUP + j) * NUP + k] = w;
+                // all loads of a thread first, then its stores: the compiler may not move a load
+                // across a store it cannot tell apart, and eight dependent round trips per layer
+                // would cost more than the group's GEMMs
+                __nv_bfloat16 wv[NUP * NUP / 128];
+#pragma unroll
+                for (int e = 0; e < NUP * NUP / 128; ++e) {
+                    const int i = tid + e * 128, j = i / NUP, k = i % NUP;
+                    wv[e] = (j < nu && k < nin) ? Wl[(size_t)(u0 + j) * K + kin0 + k] : __float2bfloat16_rn(0.0f);
                 }
-                if (tid < NUP) sh.bias_s[l][tid] = tid < nu ? m.bias[l][u0 + tid] : 0.0f;
+                const float bv = (tid < NUP && tid < nu) ? m.bias[l][u0 + tid] : 0.0f;
+                // stored source-major, [l][source k][target j]: a new activation updates all its targets
+#pragma unroll
+                for (int e = 0; e < NUP * NUP / 128; ++e) {
+                    const int i = tid + e * 128, j = i / NUP, k = i % NUP;
+                    Wg[(l * NUP + k) * NUP + j] = __bfloat162float(wv[e]);
+                }
+                if (tid < NUP) sh.bias_s[l][tid] = bv;
             }
-            for (int i = 0; i < GMAX; ++i) Nz[i * BM + row] = (valid && i < ng) ? r.noise[(size_t)smp * m.T + t0 + i] : 0.0f;
-            for (int k = 0; k < NUP; ++k) X[k * BM + row] = 0.0f;
+            {
+                float nv[GMAX];
+                const float *np = r.noise + (size_t)(valid ? smp : 0) * m.T + t0;
+#pragma unroll
+                for (int i = 0; i < GMAX; ++i) nv[i] = (valid && i < ng) ? __ldg(np + i) : 0.0f;
+#pragma unroll
+                for (int i = 0; i < GMAX; ++i) Nz[i * BM + row] = nv[i];
+            }
+            {
+                // the symbols the group's positions hold now (for the change flags), 255 where there is none
+                uint8_t xo[GMAX];
+                const uint8_t *xp = r.x + (size_t)(valid ? smp : 0) * m.T + t0;
+#pragma unroll
+                for (int i = 0; i < GMAX; ++i) xo[i] = (valid && i < ng) ? xp[i] : (uint8_t)255;
+#pragma unroll
+                for (int i = 0; i < GMAX; ++i) X[i * BM + row] = (float)xo[i];
+            }
             ep_sync();
+            if (tid == 0) trace(2);
             // ---- prefix sums out of tensor memory
             if (!mbar_wait(&sh.tfull, tf_par, r.ctl)) { dead = true; break; }
             tf_par ^= 1u;
             tc_fence_after();
+            if (tid == 0) trace(3);
             for (int l = 0; l <= L; ++l) {
                 float v[32];
                 if (sh.nu[l] > 0 && sh.kb_n[l] > 0) {
@@ -267,56 +377,59 @@ struct SweepEngine {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = 0.0f;
                 }
+                // running pre-activation of every unit of the group: prefix sum + bias; the group's own
+                // contributions are added below, each as soon as its source exists
+                const uint32_t v4 = smem_u32(V) + 4u * (uint32_t)((l * BM + row) * NUP);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) V[(l * NUP + i) * BM + row] = v[i];
+                for (int c = 0; c < NUP / 4; ++c)
+                    sts_f4(v4 + 16u * (uint32_t)(c ^ (row & 7)),
+                           make_float4(v[4 * c] + sh.bias_s[l][4 * c], v[4 * c + 1] + sh.bias_s[l][4 * c + 1],
+                                       v[4 * c + 2] + sh.bias_s[l][4 * c + 2], v[4 * c + 3] + sh.bias_s[l][4 * c + 3]));
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh.tempty);
-            // ---- the group's positions in order, thread = sample row
+            if (tid == 0) trace(4);
+            // ---- the group's positions in order, thread = sample row.  A value that becomes known (a
+            // sampled symbol, then the hidden units it completes, layer by layer) is added at once to
+            // the running sums of everything in the group that reads it: the additions of one source
+            // are independent of each other, and each target receives its sources in index order.
             for (int i = 0; i < ng; ++i) {
                 const int t = t0 + i;
-                float z = V[(L * NUP + i) * BM + row] + sh.bias_s[L][i];
-                {
-                    const float *wrow = Wg + (L * NUP + i) * NUP;
-                    const int nin = sh.nin[L];
-                    for (int k = 0; k < nin; ++k) z = fmaf(wrow[k], V[((L - 1) * NUP + k) * BM + row], z);
-                }
+                const float z = lds_f(vat(L, i, row));
                 const int xn = js_sample_binary(r.nk, z, Nz[i * BM + row]);
-                if (valid) {
-                    uint8_t *xp = r.x + (size_t)smp * m.T + t;
-                    if (*xp != (uint8_t)xn) { *xp = (uint8_t)xn; row_changed = true; }
+                if (valid && (int)X[i * BM + row] != xn) {
+                    r.x[(size_t)smp * m.T + t] = (uint8_t)xn;
+                    row_changed = true;
                 }
-                X[i * BM + row] = sh.lut_s[xn];
+                const float enc = sh.lut_s[xn];
+                X[i * BM + row] = enc;
                 if (t + 1 > hi) continue;
+                scatter(0, i, enc, row);
                 // the hidden units that position t makes computable: degree t + 1
                 for (int l = 0; l < L; ++l) {
                     const int j0 = sh.cs[l + 1][i] - sh.u0[l], j1 = sh.cs[l + 1][i + 1] - sh.u0[l];
-                    const int nin = sh.nin[l];
-                    const float *in = l == 0 ? X : V + (size_t)(l - 1) * NUP * BM;
                     for (int j = j0; j < j1; ++j) {
-                        float pre = V[(l * NUP + j) * BM + row] + sh.bias_s[l][j];
-                        const float *wrow = Wg + (l * NUP + j) * NUP;
-                        for (int k = 0; k < nin; ++k) pre = fmaf(wrow[k], in[k * BM + row], pre);
-                        V[(l * NUP + j) * BM + row] = __bfloat162float(__float2bfloat16_rn(tc_act_fn(m.act, pre)));
+                        const uint32_t pv = vat(l, j, row);
+                        const float val = __bfloat162float(__float2bfloat16_rn(tc_act_fn(m.act, lds_f(pv))));
+                        sts_f(pv, val);
+                        scatter(l + 1, j, val, row);
                     }
                 }
             }
+            if (tid == 0) trace(5);
             // ---- the group's activations into F, for the GEMMs of the groups that follow
             if (t1 < b) {
-                {
-                    __nv_bfloat16 *f = sw.F[0] + ((size_t)slot * BM + row) * sw.WF[0] + (t0 - kb_old[0] * BK);
-                    for (int i = 0; i < ng; ++i) f[i] = __float2bfloat16_rn(X[i * BM + row]);
-                }
-                for (int l = 1; l <= L; ++l) {
-                    const int n = sh.nin[l];
-                    __nv_bfloat16 *f = sw.F[l] + ((size_t)slot * BM + row) * sw.WF[l] + (sh.kin0[l] - kb_old[l] * BK);
-                    for (int j = 0; j < n; ++j) f[j] = __float2bfloat16_rn(V[((l - 1) * NUP + j) * BM + row]);
-                }
+                store_run(sw.F[0] + ((size_t)slot * BM + row) * sw.WF[0] + (t0 - kb_old[0] * BK), -1, row, ng);
+                for (int l = 1; l <= L; ++l)
+                    store_run(sw.F[l] + ((size_t)slot * BM + row) * sw.WF[l] + (sh.kin0[l] - kb_old[l] * BK), l - 1, row,
+                              sh.nin[l]);
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.gdone);
             }
+            if (tid == 0) trace(6);
+            group_no++;
         }
     }
 };
@@ -465,11 +578,11 @@ int js_sweep_prepare(js_model *mo)
         }
     }
     int G = GMAX;
-    for (; G >= 1; G >>= 1) {
+    for (; G >= 1; --G) {
         bool ok = true;
         for (int l = 1; l <= L && ok; ++l)
-            for (int d = 0; d + G <= T && ok; ++d)
-                if (cnt[l][d + G] - cnt[l][d] > NUP) ok = false;
+            for (int d = 0; d < T && ok; ++d)
+                if (cnt[l][std::min(d + G, T)] - cnt[l][d] > NUP) ok = false;
         if (ok) break;
     }
     if (G < 1) return 0;

@@ -833,6 +833,86 @@ struct TcEngine {
         return true;
     }
 
+    // ---- 256-way output layer with ONE uniform number per position (inverse CDF of the softmax):
+    // the first class c with  u * S < sum_{i<=c} e_i,  e_i = exp(z_i - max z), S their total.  The
+    // thread's 256 logits stay in tensor memory and are read three times in chunks of 32: the
+    // maximum, the running sums (remembered at the chunk ends, which tells the chunk that holds the
+    // answer), and once more for the class inside that chunk.  The running sum is carried in class
+    // order with the same instructions in the second and third reading, so both see the same values.
+    __device__ bool epi_icdf_tile(int sample, int row, int d, uint32_t tbase, const Win &w, bool flag, int parity,
+                                  bool &any_changed, int &first)
+    {
+        const float *bs = sh.bias_s[warp - 2];
+        const bool commit = sample >= 0 && d >= w.plo && d < w.phi;
+        int xold = 0;
+        float u = 0.5f;
+        if (commit) {
+            xold = (int)__ldcg(r.x + (size_t)sample * m.T + d);
+            u = __ldg(r.noise + (size_t)sample * m.T + d);
+        }
+        float mx = -INFINITY;
+#pragma unroll 1
+        for (int c0 = 0; c0 < 256; c0 += 32) {
+            uint32_t ra[32];
+            __syncwarp();
+            tmem_ld32_issue(tbase + (uint32_t)c0, ra);
+            tmem_wait_ld();
+            if (cur_parts > 0) add_partials(ra, c0);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, __uint_as_float(ra[i]) + bs[c0 + i]);
+        }
+        float run = 0.0f, cum[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            uint32_t ra[32];
+            __syncwarp();
+            tmem_ld32_issue(tbase + (uint32_t)(k * 32), ra);
+            tmem_wait_ld();
+            if (cur_parts > 0) add_partials(ra, k * 32);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) run += __expf((__uint_as_float(ra[i]) + bs[k * 32 + i]) - mx);
+            cum[k] = run;
+        }
+        const float target = u * run;
+        int ck = 8;                       // the first chunk whose closing sum exceeds the target
+        float base = 0.0f;
+#pragma unroll
+        for (int k = 7; k >= 0; --k) {
+            if (target < cum[k]) { ck = k; base = k > 0 ? cum[k - 1] : 0.0f; }
+        }
+        int bi = (run == run) ? 255 : 0;  // u at the very top of the range; no finite score: class 0
+#pragma unroll 1
+        for (int k = 0; k < 8; ++k) {
+            uint32_t ra[32];
+            __syncwarp();
+            tmem_ld32_issue(tbase + (uint32_t)(k * 32), ra);      // every lane reads (the load is warp-wide) ...
+            tmem_wait_ld();
+            if (k == 7) release_acc();
+            if (k != ck) continue;                                // ... the lanes whose answer lies elsewhere skip the rest
+            if (cur_parts > 0) add_partials(ra, k * 32);
+            float s2 = base;
+            int hit = -1;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                s2 += __expf((__uint_as_float(ra[i]) + bs[k * 32 + i]) - mx);
+                hit = (hit < 0 && target < s2) ? i : hit;
+            }
+            bi = k * 32 + (hit < 0 ? 31 : hit);
+        }
+        bool ch = false;
+        if (commit && xold != bi) {
+            r.x[(size_t)sample * m.T + d] = (uint8_t)bi;
+            ((__nv_bfloat16 *)m.a[0])[(size_t)row * m.T + d] = __float2bfloat16_rn(sh.lut_s[bi]);
+            ch = true;
+        }
+        if (flag && ch) {
+            raise_flag(parity, sample);
+            any_changed = true;
+            first = min(first, d);
+        }
+        return true;
+    }
+
     __device__ void epilogue(int l, int kind, const Win &w, bool flag, int parity, float *zout, int nt_lo,
                              int nt_hi, int MT)
     {
@@ -874,7 +954,11 @@ struct TcEngine {
             const bool owner = u.nparts >= 0;
             if (owner && kind != EPI_LOGITS) load_bias_tile(l, nt * ly.bn, ly.bn);
             int csmp = -1;
-            if (owner && kind == EPI_CAT) {
+            if (owner && kind == EPI_CAT && r.nk != JS_NOISE_GUMBEL) {
+                const int rw = mt * BM + q * 32 + lane;
+                csmp = rw < live ? perm_cur()[rw] : -1;
+            }
+            if (owner && kind == EPI_CAT && r.nk == JS_NOISE_GUMBEL) {
                 const int rw = mt * BM + q * 32 + lane;
                 csmp = rw < live ? perm_cur()[rw] : -1;
                 if (!cat_ahead) cat_prefetch(csmp, nt);          // first tile of the phase
@@ -924,7 +1008,9 @@ struct TcEngine {
                 if (!fine) { dead = true; break; }
                 if (wany) { any_changed = true; first = min(first, wfirst); }
             } else if (kind == EPI_CAT) {
-                if (!epi_cat_tile(csmp, row, nt, tbase, w, flag, parity, any_changed, first)) { dead = true; break; }
+                const bool fine = r.nk == JS_NOISE_GUMBEL ? epi_cat_tile(csmp, row, nt, tbase, w, flag, parity, any_changed, first)
+                                                          : epi_icdf_tile(csmp, row, nt, tbase, w, flag, parity, any_changed, first);
+                if (!fine) { dead = true; break; }
             } else {
                 for (int c0 = 0; c0 < ly.bn; c0 += 32) {
                     float v[32];

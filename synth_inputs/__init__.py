@@ -99,6 +99,9 @@ CONFIGS: Dict[str, object] = {
     # config 5: masked-convolution sampler
     "conv_32": ConvConfig("conv_32", 4, height=32, width=32, in_ch=3, ch=128, layers=8, C=256, batch=16),
 }
+# extension: config 3's model sampled by the categorical inverse CDF, one uniform number per position
+# (same weights: same index; 1/256 of the noise)
+CONFIGS["made_cat_icdf"] = replace(CONFIGS["made_cat"], name="made_cat_icdf", noise_kind=NOISE_UNIFORM_CAT)
 
 
 def scaled(cfg, **changes):

@@ -45,7 +45,7 @@ def run(p, cfg, model, d_noise, mode, block=0):
     return out.cpu().numpy(), iters.cpu().numpy()
 
 
-@pytest.mark.parametrize("name", ["made_784", "made_4096", "made_cat"])
+@pytest.mark.parametrize("name", ["made_784", "made_4096", "made_cat", "made_cat_icdf"])
 def test_full_size_jacobi_and_hybrids(name):
     p, cfg, orc, model, noise, d_noise, xstar = full_case(name)
     nk = cfg.noise_kind
@@ -54,17 +54,20 @@ def test_full_size_jacobi_and_hybrids(name):
     assert model.stats().path == 0, "the tensor-core kernels must serve the benchmark workloads"
     audit = check_samples(orc, x, xstar, noise, nk)
     print(f"{name}: jacobi iters mean {it.mean():.3f} max {it.max()} excused {audit}")
-    n = 12 if name != "made_cat" else 6
+    n = 12 if not name.startswith("made_cat") else 6
     ref = orc.map_batch(lambda i: orc.jacobi(noise[i], nk)[1], n, threads=16)
     clean = [i for i in range(n) if i not in audit["excused_samples"]]
     np.testing.assert_array_equal(it[clean], np.array(ref)[clean])
     assert 1 <= it.min() and it.max() <= cfg.D
-    # sequential order with the same kernels (banded)
-    model.set_option(p.JS_OPT_SEQ_SKIP, 1)
-    seq = torch.empty((cfg.batch, cfg.D), dtype=torch.uint8, device="cuda")
-    assert p.sequential_sample(model, d_noise, nk, seq) == 0
-    model.set_option(p.JS_OPT_SEQ_SKIP, 0)
-    check_samples(orc, seq.cpu().numpy(), xstar, noise, nk)
+    # sequential order: banded with the Jacobi kernels, and the library's default (the cached sweep
+    # where the model allows it)
+    for opt in (1, 2):
+        model.set_option(p.JS_OPT_SEQ_SKIP, opt)
+        seq = torch.full((cfg.batch, cfg.D), 9, dtype=torch.uint8, device="cuda")
+        t0 = time.perf_counter()
+        assert p.sequential_sample(model, d_noise, nk, seq) == 0
+        print(f"{name}: sequential_sample with JS_OPT_SEQ_SKIP={opt}: {1e3 * (time.perf_counter() - t0):.1f} ms")
+        check_samples(orc, seq.cpu().numpy(), xstar, noise, nk)
     # GS-Jacobi with the block sizes the workload names
     for B in cfg.blocks:
         x, it = run(p, cfg, model, d_noise, p.JS_GS_JACOBI, B)

@@ -90,8 +90,17 @@ CAT_ROWS = si.scaled(si.CONFIGS["made_cat"], D=16, H=(64, 64), batch=100)
 # uniform noise with the inverse-CDF rule on a bf16 model (the tensor-core epilogue has one instance per noise kind)
 BIN_ICDF = si.scaled(si.CONFIGS["made_784"], D=144, H=(128,), batch=40, noise_kind=si.NOISE_UNIFORM_ICDF)
 
+# 256-way positions sampled by the inverse CDF of the softmax from one uniform number each; the second
+# case has long K ranges, so the tensor-core kernels cut its output tiles into several work units
+CAT_ICDF = si.scaled(si.CONFIGS["made_cat"], D=24, H=(128, 96), batch=70, noise_kind=si.NOISE_UNIFORM_CAT, index=7)
+CAT_ICDF_SPLIT = si.scaled(si.CONFIGS["made_cat"], D=16, H=(2688,), batch=20, noise_kind=si.NOISE_UNIFORM_CAT,
+                           index=8, w_var_scale=2.0)
+# 7-way positions: CUDA-core kernels only
+CAT7_ICDF = si.MadeConfig("cat7", 9, D=20, C=7, H=(48,), act=si.ACT_RELU, prec=si.PREC_F32, batch=11,
+                          noise_kind=si.NOISE_UNIFORM_CAT, w_var_scale=8.0, b_var=0.2)
+
 CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN, "split": SPLIT, "cat_rows": CAT_ROWS,
-         "bin_icdf": BIN_ICDF}
+         "bin_icdf": BIN_ICDF, "cat_icdf": CAT_ICDF, "cat_icdf_split": CAT_ICDF_SPLIT, "cat7_icdf": CAT7_ICDF}
 # kernel path: 1 = CUDA-core kernels, 0 = tensor-core kernels (bf16 models only)
 COMBOS = [(n, 1) for n in CASES] + [(n, 0) for n in CASES if n != "tiny"]
 COMBO_IDS = [f"{n}-{'tc' if p == 0 else 'cc'}" for n, p in COMBOS]
@@ -174,7 +183,8 @@ def test_sequential_and_gauss_seidel(name, seq_skip):
 
 
 @pytest.mark.parametrize("name,blocks", [("tiny", (1, 4, 5, 16)), ("bin", (64, 30, 1, 200)), ("cat", (8, 5)),
-                                         ("chain", (32, 64, 100)), ("split", (256,)), ("bin_icdf", (48,))])
+                                         ("chain", (32, 64, 100)), ("split", (256,)), ("bin_icdf", (48,)),
+                                         ("cat_icdf", (8,)), ("cat7_icdf", (6,))])
 @pytest.mark.parametrize("skip", [1, 0])
 def test_hybrids(name, blocks, skip):
     _skip_if_not_applicable(name)
