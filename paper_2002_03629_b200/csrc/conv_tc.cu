@@ -33,6 +33,10 @@ constexpr int SMEM_BYTES = RING_BYTES + STAGING_BYTES + 1024;
 constexpr int MAX_IMAGES = 256;
 
 enum { EPI_HIDDEN = 0, EPI_LOGITS = 1, EPI_CAT = 3 };
+// which activations a layer reads and writes.  SRC_NEW: the working set.  SRC_OLD: the set of the previous
+// outer iterate (Jacobi-GS).  SRC_MIXED: the row above from the previous outer iterate, the own row from
+// the working set - the view a one-row block has in Algorithm 2.
+enum { SRC_NEW = 0, SRC_OLD = 1, SRC_MIXED = 2 };
 
 // the five taps a causal 3x3 kernel keeps, in the order the packed weights use
 __device__ __constant__ int c_tap_ky[5] = {0, 0, 0, 1, 1};
@@ -48,7 +52,7 @@ struct ConvShared {
 };
 
 struct ConvEngine {
-    static constexpr bool has_jgs = false;
+    static constexpr bool has_jgs = true;
     const ConvDev &m;
     const RunArgs &r;
     ConvShared &sh;
@@ -179,12 +183,12 @@ struct ConvEngine {
         return l < m.n_conv ? 5 * (m.cin_pad[l] / BK) : m.ch / BK;
     }
 
-    __device__ void producer(int l, int yt_lo, int nyl, int ntiles)
+    __device__ void producer(int l, int yt_lo, int nyl, int ntiles, int src)
     {
         const bool head = (l == m.n_conv);
         const int per = head ? m.in_ch : 1;
         const int bn = head ? 256 : m.ch;
-        const CUtensorMap *ma = m.tmAct + l, *mw = m.tmW + l;
+        const CUtensorMap *ma_new = m.tmAct + l, *ma_old = m.tmActOld + l, *mw = m.tmW + l;
         const uint32_t bytes = A_BYTES + bn * BK * 2;
         const int kcs = head ? m.ch / BK : m.cin_pad[l] / BK;
         trace(0);
@@ -195,6 +199,7 @@ struct ConvEngine {
             const int ntaps = head ? 1 : 5;
             for (int tap = 0; tap < ntaps && !dead; ++tap) {
                 const int dy = head ? 0 : c_tap_ky[tap] - 1, dx = head ? 0 : c_tap_kx[tap] - 1;
+                const CUtensorMap *ma = (src == SRC_OLD || (src == SRC_MIXED && dy < 0)) ? ma_old : ma_new;
                 for (int kc = 0; kc < kcs; ++kc) {
                     if (!mbar_wait(&sh.empty[stage], sphase ^ 1u, r.ctl)) { dead = true; break; }
                     mbar_expect_tx(&sh.full[stage], bytes);
@@ -245,7 +250,7 @@ struct ConvEngine {
 
     // conv layer: ReLU(acc + bias) -> bf16, through the staging buffer so that the NHWC stores
     // are coalesced (see the masked-MLP kernel for the layout of the staging rows)
-    __device__ void epi_hidden_tile(int l, int n, int y0, uint32_t tbase)
+    __device__ void epi_hidden_tile(int l, int n, int y0, uint32_t tbase, int src)
     {
         uint8_t *stg = staging + (size_t)(warp - 2) * 8192;
         const float *bs = sh.bias_s[warp - 2];
@@ -266,7 +271,7 @@ struct ConvEngine {
             }
         }
         release_acc();
-        __nv_bfloat16 *out = (__nv_bfloat16 *)m.act[l + 1];
+        __nv_bfloat16 *out = (__nv_bfloat16 *)(src == SRC_OLD ? m.act_old[l + 1] : m.act[l + 1]);
         const int q = warp & 3, ch = lane & 15;
         const int col = ch * 8;
         const int rows_valid = (min(m.height, y0 + m.R) - y0) * m.width;     // pixels of the tile inside the image
@@ -282,7 +287,7 @@ struct ConvEngine {
     }
 
     __device__ void epilogue(int l, int kind, const Win &w, bool flag, int parity, float *zout, int yt_lo, int nyl,
-                             int ntiles)
+                             int ntiles, int src)
     {
         const bool head = (l == m.n_conv);
         const int per = head ? m.in_ch : 1;
@@ -304,7 +309,7 @@ struct ConvEngine {
             if (warp == 4 && lane == 0) trace(3);
             const uint32_t tbase = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * ACC_COLS);
             if (!head) {
-                epi_hidden_tile(l, n, y0, tbase);
+                epi_hidden_tile(l, n, y0, tbase, src);
             } else {
                 // thread = one pixel of the tile; 256 logits of sub-pixel c
                 const int prow = q * 32 + lane;
@@ -381,7 +386,7 @@ struct ConvEngine {
         }
     }
 
-    __device__ bool layer_phase(int l, int kind, const Win &w, bool flag, int parity, float *zout)
+    __device__ bool layer_phase(int l, int kind, const Win &w, bool flag, int parity, float *zout, int src = SRC_NEW)
     {
         const bool head = (l == m.n_conv);
         int yt_lo, yt_hi;
@@ -401,24 +406,82 @@ struct ConvEngine {
         if (ntiles == 0) return false;
         phase_no++;
         if (warp == 0) {
-            if (lane == 0) producer(l, yt_lo, nyl, ntiles);
+            if (lane == 0) producer(l, yt_lo, nyl, ntiles, src);
         } else if (warp == 1) {
             if (lane == 0) mma_issuer(l, ntiles);
         } else {
-            epilogue(l, kind, w, flag, parity, zout, yt_lo, nyl, ntiles);
+            epilogue(l, kind, w, flag, parity, zout, yt_lo, nyl, ntiles, src);
         }
         return true;
     }
 
-    __device__ bool step(const Win &w, bool flag, int parity, float *zout)
+    __device__ bool step(const Win &w, bool flag, int parity, float *zout, int src = SRC_NEW)
     {
-        for (int l = 0; l <= m.n_conv; ++l) {
+        const int l_end = src == SRC_OLD ? m.n_conv - 1 : m.n_conv;      // the old set needs no head
+        for (int l = 0; l <= l_end; ++l) {
             const bool last = (l == m.n_conv);
-            const bool did = layer_phase(l, last ? (zout ? EPI_LOGITS : EPI_CAT) : EPI_HIDDEN, w, last && flag, parity, zout);
-            if (did || last)
+            const bool did = layer_phase(l, last ? (zout ? EPI_LOGITS : EPI_CAT) : EPI_HIDDEN, w, last && flag, parity, zout, src);
+            if (did || l == l_end)
                 if (!barrier()) return false;
         }
         return true;
+    }
+
+    // One outer iteration of Algorithm 2 with one-image-row blocks.  A block's sequential sweep yields the
+    // unique solution of the block's own triangular system given the rows above at the previous outer
+    // iterate; Jacobi iterations on that sub-system reach the very same solution in at most |B| steps
+    // (Proposition 1 applied to the block), and they can run for all rows of all images at once as
+    // forward passes in which every layer reads the row above from the activations of x^{k-1} and its
+    // own row from the working activations.  So: the hidden layers once on x^{k-1} (the "old" set),
+    // then mixed passes until no symbol changes, then the comparison with x^{k-1} for the outer flags,
+    // which are left in the flag slot `parity`.
+    __device__ bool jgs_outer(int parity, int, int, int &iterations)
+    {
+        const size_t n = (size_t)r.batch * m.T;
+        const size_t npix64 = (size_t)r.batch * m.height * m.width * 64 / 8;       // uint4 units of the padded image
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+            r.x_old[i] = r.x[i];
+        {
+            const uint4 *src = reinterpret_cast<const uint4 *>(m.act[0]);
+            uint4 *dst = reinterpret_cast<uint4 *>(m.act_old[0]);
+            for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < npix64; i += (size_t)gridDim.x * blockDim.x)
+                dst[i] = src[i];
+        }
+        if (!barrier()) return false;
+        // every CTA has read the previous outer iteration's flags by now: both slots start clean
+        if (blockIdx.x == 0) {
+            for (int i = threadIdx.x; i < 2 * r.batch; i += blockDim.x) r.smp_changed[i] = 0;
+            if (threadIdx.x == 0) {
+                r.ctl->agg_any[0] = r.ctl->agg_any[1] = 0;
+                r.ctl->agg_minfirst[0] = r.ctl->agg_minfirst[1] = INT_MAX;
+            }
+        }
+        const Win w = make_win(0, m.T, 0, m.T);
+        if (!step(w, false, 0, nullptr, SRC_OLD)) return false;
+        iterations++;
+        const int cap = m.width * m.in_ch;
+        int q = parity;
+        for (int k = 1; k <= cap; ++k) {
+            q ^= 1;
+            if (!step(w, true, q, nullptr, SRC_MIXED)) return false;
+            iterations++;
+            const int any = ld_volatile_i32(&r.ctl->agg_any[q]);
+            reset_other_parity(r, q);
+            if (!barrier()) return false;
+            if (!any) break;
+        }
+        // both flag slots start clean, then the outer comparison fills slot `parity`
+        if (blockIdx.x == 0) {
+            for (int i = threadIdx.x; i < 2 * r.batch; i += blockDim.x) r.smp_changed[i] = 0;
+            if (threadIdx.x == 0) {
+                r.ctl->agg_any[0] = r.ctl->agg_any[1] = 0;
+                r.ctl->agg_minfirst[0] = r.ctl->agg_minfirst[1] = INT_MAX;
+            }
+        }
+        if (!barrier()) return false;
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+            if (r.x[i] != r.x_old[i]) note_change(r, parity, (int)(i / m.T), (int)(i % m.T));
+        return barrier();
     }
 };
 
@@ -524,18 +587,21 @@ int js_conv_build(js_model *mo, const js_conv_desc *d)
     const size_t npix = (size_t)nb * d->height * d->width;
     auto group = [&](int k) { return (int)(((long long)d->in_ch * k) / ch); };
 
-    std::vector<CUtensorMap> mapsA(d->n_conv + 1), mapsW(d->n_conv + 1);
+    std::vector<CUtensorMap> mapsA(d->n_conv + 1), mapsAold(d->n_conv + 1), mapsW(d->n_conv + 1);
     for (int l = 0; l <= d->n_conv; ++l) {
         const int c_l = l == 0 ? 64 : ch;                 // channels of act[l] (the image is padded to 64)
         if (l < d->n_conv) v.cin_pad[l] = c_l;
-        __nv_bfloat16 *a = nullptr;
-        if (!upload<__nv_bfloat16>(mo, nullptr, npix * c_l, &a)) return JS_ERR_CUDA;
-        v.act[l] = a;
-        const cuuint64_t dims[4] = {(cuuint64_t)c_l, (cuuint64_t)d->width, (cuuint64_t)d->height, (cuuint64_t)nb};
-        const cuuint64_t strides[3] = {(cuuint64_t)c_l * 2, (cuuint64_t)d->width * c_l * 2,
-                                       (cuuint64_t)d->height * d->width * c_l * 2};
-        const cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)d->width, (cuuint32_t)v.R, 1};
-        if (!encode_nd(&mapsA[l], a, 4, dims, strides, box)) return JS_ERR_UNSUPPORTED;
+        // two sets: the working activations, and those of the previous outer iterate (Jacobi-GS)
+        for (int set = 0; set < 2; ++set) {
+            __nv_bfloat16 *a = nullptr;
+            if (!upload<__nv_bfloat16>(mo, nullptr, npix * c_l, &a)) return JS_ERR_CUDA;
+            (set == 0 ? v.act[l] : v.act_old[l]) = a;
+            const cuuint64_t dims[4] = {(cuuint64_t)c_l, (cuuint64_t)d->width, (cuuint64_t)d->height, (cuuint64_t)nb};
+            const cuuint64_t strides[3] = {(cuuint64_t)c_l * 2, (cuuint64_t)d->width * c_l * 2,
+                                           (cuuint64_t)d->height * d->width * c_l * 2};
+            const cuuint32_t box[4] = {(cuuint32_t)BK, (cuuint32_t)d->width, (cuuint32_t)v.R, 1};
+            if (!encode_nd(set == 0 ? &mapsA[l] : &mapsAold[l], a, 4, dims, strides, box)) return JS_ERR_UNSUPPORTED;
+        }
     }
     static const int tky[5] = {0, 0, 0, 1, 1}, tkx[5] = {0, 1, 2, 0, 1};
     for (int l = 0; l < d->n_conv; ++l) {
@@ -586,7 +652,9 @@ int js_conv_build(js_model *mo, const js_conv_desc *d)
         if (!upload<float>(mo, lut.data(), lut.size(), &ld)) return JS_ERR_CUDA;
         v.lut = ld;
     }
-    CUtensorMap *pa = nullptr, *pw = nullptr;
+    CUtensorMap *pa = nullptr, *pw = nullptr, *pao = nullptr;
+    if (!upload<CUtensorMap>(mo, mapsAold.data(), mapsAold.size(), &pao)) return JS_ERR_CUDA;
+    v.tmActOld = pao;
     if (!upload<CUtensorMap>(mo, mapsA.data(), mapsA.size(), &pa)) return JS_ERR_CUDA;
     if (!upload<CUtensorMap>(mo, mapsW.data(), mapsW.size(), &pw)) return JS_ERR_CUDA;
     v.tmAct = pa;

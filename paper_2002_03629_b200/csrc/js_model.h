@@ -57,9 +57,11 @@ struct ConvDev {
     int nyt;                            // row tiles per image
     int cin_pad[JS_MAXL];               // input channels of conv layer l, padded to a multiple of 64
     void *act[JS_MAXL + 1];             // NHWC bf16; act[0] = encoded image padded to 64 channels
+    void *act_old[JS_MAXL + 1];         // the same for the previous outer iterate (Jacobi-GS)
     const float *bias[JS_MAXL + 1];     // conv biases, head bias at [n_conv]
     const float *lut;
     const CUtensorMap *tmAct;           // [n_conv+1] 4-D maps {channel, x, y, image}, box 64 x width x R x 1
+    const CUtensorMap *tmActOld;        // the same over act_old
     const CUtensorMap *tmW;             // [n_conv+1] 2-D maps of the packed weights
 };
 

@@ -124,9 +124,32 @@ def test_conv_max_iters_and_unsupported_mode():
     clean = [s for s in range(cfg.batch) if s not in audit["excused_samples"]]
     np.testing.assert_array_equal(x[clean], ref[clean])
     assert len(clean) >= cfg.batch - 1
+    # Algorithm 2 is served for blocks of one image row only
     with pytest.raises(p.JsError) as e:
-        c.run(p.JS_JACOBI_GS, block=48)
+        c.run(p.JS_JACOBI_GS, block=40)
     assert e.value.code == p.JS_ERR_UNSUPPORTED
+
+
+def test_conv_jacobi_gs_one_row_blocks():
+    """Algorithm 2 with one-image-row blocks (Section 5.3.2): samples equal the feedforward pass, outer
+    iteration counts equal the oracle's, also from a random start and under a lowered cap."""
+    c = small()
+    p, cfg = c.p, c.cfg
+    B = cfg.width * cfg.in_ch
+    for init in (None, si.random_init(cfg, salt=4)):
+        rc, x, it = c.run(p.JS_JACOBI_GS, block=B, init=init)
+        assert rc == 0
+        audit = check_samples(c.orc, x, c.xstar, c.noise, c.nk)
+        ref = [c.orc.jacobi_gs(c.noise[s], c.nk, B, None if init is None else init[s])[1] for s in range(cfg.batch)]
+        clean = [s for s in range(cfg.batch) if s not in audit["excused_samples"]]
+        np.testing.assert_array_equal(it[clean], np.array(ref)[clean])
+        assert max(ref) >= 3, "the small conv case should need a few outer iterations"
+    rc, x, it = c.run(p.JS_JACOBI_GS, block=B, max_iters=2)
+    assert rc == p.JS_NOT_CONVERGED and np.all(it == 2)
+    ref = np.stack([c.orc.jacobi_gs(c.noise[s], c.nk, B, None, 2)[0] for s in range(cfg.batch)])
+    audit = check_samples(c.orc, x, c.xstar, c.noise, c.nk, hi=2 * B)       # two rows are final (Proposition 2)
+    clean = [s for s in range(cfg.batch) if s not in audit["excused_samples"]]
+    np.testing.assert_array_equal(x[clean], ref[clean])
 
 
 def torch_top_hidden_max(cfg, W, b, lut, x):
@@ -280,3 +303,13 @@ def test_conv_full_size_config():
     assert rc == 0
     np.testing.assert_array_equal(x2, x)
     print(f"conv_32: gs-jacobi (2 rows) inner iterations mean {it2.mean():.1f}")
+    import time
+    t0 = time.perf_counter()
+    rc, x3, it3 = c.run(p.JS_JACOBI_GS, block=cfg.width * cfg.in_ch)
+    dt = time.perf_counter() - t0
+    assert rc == 0
+    np.testing.assert_array_equal(x3, x)
+    ref3 = np.array(c.orc.map_batch(lambda i: c.orc.jacobi_gs(c.noise[i], c.nk, cfg.width * cfg.in_ch)[1], 4, threads=4))
+    print(f"conv_32: jacobi-gs (one-row blocks) {1e3 * dt:.1f} ms, outer iterations {it3.tolist()}, oracle (first four) "
+          f"{ref3.tolist()}, forward passes {c.model.stats().iterations}")
+    assert np.abs(it3[:4] - ref3).max() <= 2
