@@ -46,7 +46,7 @@ typedef enum { JS_JACOBI = 0, JS_GAUSS_SEIDEL = 1, JS_GS_JACOBI = 2, JS_JACOBI_G
  *   GUMBEL        x = argmax_c (z_c + g_c)  noise [batch][T][C]   Gumbel(0,1), lowest index wins ties
  *   UNIFORM_CAT   x = first class c with u < F_c, F_c = sum_{i<=c} softmax(z)_i (inverse CDF of a C-way
  *                 position)                 noise [batch][T]      in (0,1); one number per position, so
- *                 1/C of the noise bytes of GUMBEL; masked MLPs only */
+ *                 1/C of the noise bytes of GUMBEL */
 typedef enum { JS_NOISE_UNIFORM_ICDF = 0, JS_NOISE_LOGISTIC = 1, JS_NOISE_GUMBEL = 2, JS_NOISE_UNIFORM_CAT = 3 } js_noise_kind;
 typedef enum { JS_ACT_RELU = 0, JS_ACT_GELU_TANH = 1 } js_act;
 /* JS_F32: fp32 weights and activations.  JS_BF16: weights rounded to bf16 after

@@ -196,6 +196,52 @@ class Oracle:
         fn = lib().orc_jacobi_gs_literal if literal else lib().orc_jacobi_gs
         return self._hybrid(fn, noise, nk, init, block, max_iters)
 
+    # ---- continuous states (C == 2: location and log-scale per position) ----
+    def _real(self, a, n):
+        a = np.ascontiguousarray(a, dtype=np.float32)
+        assert a.shape == (n,), a.shape
+        return a
+
+    def forward_logits_real(self, x: np.ndarray) -> np.ndarray:
+        assert self.C == 2
+        x = self._real(x, self.T)
+        z = np.empty((self.T, 2), dtype=np.float32)
+        lib().orc_forward_logits_real(self._h, _fptr(x), _fptr(z))
+        return z
+
+    def jacobi_step_real(self, x: np.ndarray, noise: np.ndarray) -> np.ndarray:
+        x, noise = self._real(x, self.T), self._real(noise, self.T)
+        out = np.empty(self.T, dtype=np.float32)
+        lib().orc_jacobi_step_real(self._h, _fptr(x), _fptr(noise), _fptr(out))
+        return out
+
+    def sequential_real(self, noise: np.ndarray) -> np.ndarray:
+        noise = self._real(noise, self.T)
+        x = np.empty(self.T, dtype=np.float32)
+        lib().orc_sequential_real(self._h, _fptr(noise), _fptr(x))
+        return x
+
+    def jacobi_real(self, noise: np.ndarray, eps: float = 0.0, init: Optional[np.ndarray] = None, max_iters: int = 0):
+        """Algorithm 1 on continuous states.  Returns (x, iters, converged)."""
+        noise = self._real(noise, self.T)
+        init = None if init is None else self._real(init, self.T)
+        x = np.empty(self.T, dtype=np.float32)
+        it, cv = C.c_int(0), C.c_int(0)
+        lib().orc_jacobi_real(self._h, _fptr(noise), None if init is None else _fptr(init), C.c_float(eps), max_iters,
+                              _fptr(x), C.byref(it), C.byref(cv))
+        return x, it.value, bool(cv.value)
+
+    def gs_jacobi_real(self, noise: np.ndarray, block: int, eps: float = 0.0, init: Optional[np.ndarray] = None,
+                       max_iters: int = 0):
+        """Algorithm 3 on continuous states.  Returns (x, summed inner iterations, converged)."""
+        noise = self._real(noise, self.T)
+        init = None if init is None else self._real(init, self.T)
+        x = np.empty(self.T, dtype=np.float32)
+        it, cv = C.c_int(0), C.c_int(0)
+        lib().orc_gs_jacobi_real(self._h, _fptr(noise), None if init is None else _fptr(init), block, C.c_float(eps),
+                                 max_iters, _fptr(x), C.byref(it), C.byref(cv))
+        return x, it.value, bool(cv.value)
+
     # ---- batches ---------------------------------------------------------
     def map_batch(self, fn, n: int, threads: int = 1):
         """Run ``fn(i)`` for i in range(n), on a thread pool if threads > 1."""

@@ -680,3 +680,115 @@ void orc_jacobi_gs_literal(const orc_model *m, const float *noise, int nk, const
     if (converged) *converged = (same || k == M) ? 1 : 0;
     free(prev); free(y); free(z);
 }
+
+/* ------------------------------------------------- continuous states (masked MLP)
+ * The paper's MADE has logistic conditionals (Section 5.3.1, Appendix C.3): every state x_t is a real
+ * number, the network reads the states themselves and gives position t two numbers, a location m_t
+ * and a log-scale l_t, from x_{<t}; with the uniform number u_t reserved for the position (Appendix
+ * A.3) the inverse CDF of the logistic law gives  x_t = m_t + exp(l_t) * logit(u_t).  The noise
+ * passed in is logit(u_t) already (the same array as for binary positions with logistic noise).
+ * C must be 2: logit 2t is m_t, logit 2t+1 is l_t.  In a bf16 model the inputs are rounded to bf16
+ * like any activation.  States are floats; the update is evaluated in double and rounded once.
+ */
+static void made_forward_real(const orc_model *m, const float *x, float *z)
+{
+    made_ws ws; made_ws_alloc(m, &ws);
+    for (int d = 0; d < m->T; ++d) ws.a[0][d] = m->prec == ORC_PREC_BF16 ? round_bf16(x[d]) : x[d];
+    for (int l = 0; l < m->L; ++l)
+        for (int i = 0; i < m->n[l + 1]; ++i)
+            ws.a[l + 1][i] = hidden_value(m->act, m->prec, made_unit(m, l, i, ws.a[l]));
+    for (int i = 0; i < m->n[m->L + 1]; ++i) z[i] = (float)made_unit(m, m->L, i, ws.a[m->L]);
+    made_ws_free(m, &ws);
+}
+
+void orc_forward_logits_real(const orc_model *m, const float *x, float *z) { made_forward_real(m, x, z); }
+
+static float real_state(const float *zt, float eps_t)
+{
+    return (float)((double)zt[0] + exp((double)zt[1]) * (double)eps_t);
+}
+
+/* one parallel update of all positions (inner loop of Algorithm 1) */
+void orc_jacobi_step_real(const orc_model *m, const float *x_in, const float *noise, float *x_out)
+{
+    float *z = (float *)malloc(sizeof(float) * (size_t)m->T * 2);
+    made_forward_real(m, x_in, z);
+    for (int t = 0; t < m->T; ++t) x_out[t] = real_state(z + 2 * t, noise[t]);
+    free(z);
+}
+
+/* Eq. 1 in the plainest form: for each t a complete forward pass on the current x, of which position t is kept */
+void orc_sequential_real(const orc_model *m, const float *noise, float *x)
+{
+    float *z = (float *)malloc(sizeof(float) * (size_t)m->T * 2);
+    for (int t = 0; t < m->T; ++t) x[t] = 0.0f;
+    for (int t = 0; t < m->T; ++t) {
+        made_forward_real(m, x, z);
+        x[t] = real_state(z + 2 * t, noise[t]);
+    }
+    free(z);
+}
+
+/*
+ * Algorithm 1 with the stopping rule of Section 2.2.1: x^0 = init (zeros if NULL); repeat k <- k+1,
+ * x^k = G(x^{k-1}) until k == cap or max_t |x^k_t - x^{k-1}_t| <= eps (the paper leaves the norm open
+ * and stops its image samplers on the largest deviation, Section 5.3.2: the maximum norm here).
+ * cap = T, lowered to max_iters when 0 < max_iters < T.  *converged is 1 when the forward difference
+ * test fired or k reached T (Proposition 1: exact then).
+ */
+void orc_jacobi_real(const orc_model *m, const float *noise, const float *init, float eps, int max_iters,
+                     float *x, int *iters, int *converged)
+{
+    int T = m->T;
+    int cap = (max_iters > 0 && max_iters < T) ? max_iters : T;
+    float *prev = (float *)malloc(sizeof(float) * (size_t)T);
+    for (int t = 0; t < T; ++t) x[t] = init ? init[t] : 0.0f;
+    int k = 0, stop = 0;
+    do {
+        k += 1;
+        memcpy(prev, x, sizeof(float) * (size_t)T);
+        orc_jacobi_step_real(m, prev, noise, x);
+        float dmax = 0.0f;
+        for (int t = 0; t < T; ++t) {
+            float d = fabsf(x[t] - prev[t]);
+            if (!(d <= dmax)) dmax = d;                 /* a NaN difference counts as a change */
+        }
+        stop = dmax <= eps;
+    } while (k < cap && !stop);
+    if (iters) *iters = k;
+    if (converged) *converged = (stop || k == T) ? 1 : 0;
+    free(prev);
+}
+
+/* Algorithm 3 on continuous states: blocks in order, Jacobi inside block [a, b) until k == |B_i| or the
+ * block's largest change is <= eps; the block starts from init.  *iters = sum of inner iterations. */
+void orc_gs_jacobi_real(const orc_model *m, const float *noise, const float *init, int block, float eps,
+                        int max_iters, float *x, int *iters, int *converged)
+{
+    int T = m->T;
+    float *next = (float *)malloc(sizeof(float) * (size_t)T);
+    for (int t = 0; t < T; ++t) x[t] = init ? init[t] : 0.0f;
+    int total = 0, conv_all = 1;
+    for (int a = 0; a < T; a += block) {
+        int b = a + block < T ? a + block : T;
+        int len = b - a;
+        int cap = (max_iters > 0 && max_iters < len) ? max_iters : len;
+        int k = 0, stop = 0;
+        do {
+            k += 1;
+            orc_jacobi_step_real(m, x, noise, next);
+            float dmax = 0.0f;
+            for (int t = a; t < b; ++t) {
+                float d = fabsf(next[t] - x[t]);
+                if (!(d <= dmax)) dmax = d;
+            }
+            stop = dmax <= eps;
+            memcpy(x + a, next + a, sizeof(float) * (size_t)len);
+        } while (k < cap && !stop);
+        total += k;
+        if (!(stop || k == len)) conv_all = 0;
+    }
+    if (iters) *iters = total;
+    if (converged) *converged = conv_all;
+    free(next);
+}

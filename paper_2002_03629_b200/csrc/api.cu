@@ -342,7 +342,6 @@ int run_made(js_model *m, RunArgs &r, cudaStream_t st)
     const MadeDev &v = m->made;
     // Algorithm 2 on the masked-conv stack: blocks of one image row (the paper's choice, Section 5.3.2)
     if (m->kind == 1 && r.kmode == KM_JACOBI_GS && r.block != m->conv.width * m->conv.in_ch) return JS_ERR_UNSUPPORTED;
-    if (m->kind == 1 && r.nk == JS_NOISE_UNIFORM_CAT && r.kmode != KM_FORWARD) return JS_ERR_UNSUPPORTED;
     // the sweeps: the strict order with cached hidden units, and Algorithm 2
     if (r.kmode == KM_SEQ && m->opt_seq_skip == 2 && sweeps_usable(m, r)) return run_sweep_sequential(m, r, st);
     if (r.kmode == KM_JACOBI_GS && sweeps_usable(m, r)) return run_jacobi_gs_tc(m, r, st);

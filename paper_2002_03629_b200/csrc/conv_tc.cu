@@ -286,6 +286,54 @@ struct ConvEngine {
         __syncwarp();
     }
 
+    // Inverse CDF of the softmax from one uniform number u: the first class c with u * S < sum_{i<=c} e_i,
+    // e_i = exp(z_i - max z).  Three readings of the thread's 256 logits out of tensor memory: the maximum,
+    // the running sums (kept at the chunk ends), the class inside the chunk found.  Kept out of line: it
+    // must not cost the Gumbel path registers.
+    __device__ __noinline__ int head_icdf(uint32_t tbase, const float *bias, float u)
+    {
+        float mx = -INFINITY;
+        for (int c0 = 0; c0 < 256; c0 += 32) {
+            float v[32];
+            __syncwarp();
+            tmem_ld32(tbase + (uint32_t)c0, v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, v[i] + __ldg(bias + c0 + i));
+        }
+        float run = 0.0f, cum[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            float v[32];
+            __syncwarp();
+            tmem_ld32(tbase + (uint32_t)(k * 32), v);
+#pragma unroll
+            for (int i = 0; i < 32; ++i) run += __expf((v[i] + __ldg(bias + k * 32 + i)) - mx);
+            cum[k] = run;
+        }
+        const float target = u * run;
+        int ck = 8;
+        float base = 0.0f;
+#pragma unroll
+        for (int k = 7; k >= 0; --k)
+            if (target < cum[k]) { ck = k; base = k > 0 ? cum[k - 1] : 0.0f; }
+        int bi = (run == run) ? 255 : 0;          // u at the very top of the range; no finite score: class 0
+        for (int k = 0; k < 8; ++k) {
+            float v[32];
+            __syncwarp();
+            tmem_ld32(tbase + (uint32_t)(k * 32), v);         // warp-wide load: every lane takes part
+            if (k != ck) continue;
+            float s2 = base;
+            int hit = -1;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                s2 += __expf((v[i] + __ldg(bias + k * 32 + i)) - mx);
+                hit = (hit < 0 && target < s2) ? i : hit;
+            }
+            bi = k * 32 + (hit < 0 ? 31 : hit);
+        }
+        return bi;
+    }
+
     __device__ void epilogue(int l, int kind, const Win &w, bool flag, int parity, float *zout, int yt_lo, int nyl,
                              int ntiles, int src)
     {
@@ -325,6 +373,9 @@ struct ConvEngine {
                 const bool commit = kind == EPI_CAT && valid && t >= w.plo && t < w.phi;
                 int xold = 0;
                 if (commit) xold = (int)__ldcg(r.x + at);
+                if (kind == EPI_CAT && r.nk == JS_NOISE_UNIFORM_CAT) {
+                    bi = head_icdf(tbase, bias, commit ? __ldg(r.noise + at) : 0.5f);
+                } else
                 for (int c0 = 0; c0 < 256; c0 += 32) {
                     float v[32];
                     __syncwarp();

@@ -313,3 +313,25 @@ def test_conv_full_size_config():
     print(f"conv_32: jacobi-gs (one-row blocks) {1e3 * dt:.1f} ms, outer iterations {it3.tolist()}, oracle (first four) "
           f"{ref3.tolist()}, forward passes {c.model.stats().iterations}")
     assert np.abs(it3[:4] - ref3).max() <= 2
+
+
+def test_conv_inverse_cdf_sampling():
+    """The head's 256-way positions sampled by the inverse CDF of the softmax from one uniform number each:
+    Jacobi, the sequential order and Jacobi-GS against the oracle's feedforward pass."""
+    cfg = si.scaled(SMALL, noise_kind=si.NOISE_UNIFORM_CAT, index=62)
+    c = ConvCase(cfg, gain=2.0)
+    p = c.p
+    assert c.noise.shape == (cfg.batch, cfg.D)
+    rc, x, it = c.run(p.JS_JACOBI)
+    assert rc == 0
+    audit = check_samples(c.orc, x, c.xstar, c.noise, c.nk)
+    ref = [c.orc.jacobi(c.noise[s], c.nk)[1] for s in range(cfg.batch)]
+    clean = [s for s in range(cfg.batch) if s not in audit["excused_samples"]]
+    np.testing.assert_array_equal(it[clean], np.array(ref)[clean])
+    assert max(ref) > 3
+    out = torch.empty((cfg.batch, cfg.D), dtype=torch.uint8, device="cuda")
+    assert p.sequential_sample(c.model, c.d_noise, c.nk, out) == 0
+    check_samples(c.orc, out.cpu().numpy(), c.xstar, c.noise, c.nk)
+    rc, x2, it2 = c.run(p.JS_JACOBI_GS, block=cfg.width * cfg.in_ch)
+    assert rc == 0
+    check_samples(c.orc, x2, c.xstar, c.noise, c.nk)

@@ -36,6 +36,11 @@ MUTANTS = [
      "for (int c = 0; c < C; ++c) { cum[c] = run; run += exp((double)nz[c] - mx); }"),
     ("softmax without the logits' scale", "run += exp((double)nz[c] - mx); cum[c] = run; }", "run += exp(0.5 * ((double)nz[c] - mx)); cum[c] = run; }"),
     ("custom degrees ignored", "? hidden_deg[l - 1][j]", "? 1 + (int)(((long long)j * (T - 1)) / m->n[l])"),
+    ("continuous state: log-scale used as the scale", "(double)zt[0] + exp((double)zt[1]) * (double)eps_t", "(double)zt[0] + (double)zt[1] * (double)eps_t"),
+    ("continuous state: noise subtracted", "(double)zt[0] + exp((double)zt[1]) * (double)eps_t", "(double)zt[0] - exp((double)zt[1]) * (double)eps_t"),
+    ("continuous state: mean change instead of the largest", "            if (!(d <= dmax)) dmax = d;                 /* a NaN difference counts as a change */", "            dmax += d / (float)T;"),
+    ("continuous state: bf16 model reads unrounded inputs", "ws.a[0][d] = m->prec == ORC_PREC_BF16 ? round_bf16(x[d]) : x[d];", "ws.a[0][d] = x[d];"),
+    ("continuous state: GS-Jacobi looks at the whole iterate", "            for (int t = a; t < b; ++t) {\n                float d = fabsf(next[t] - x[t]);", "            for (int t = 0; t < T; ++t) {\n                float d = fabsf(next[t] - x[t]);"),
 ]
 
 
@@ -50,7 +55,8 @@ def _run_mutant(case):
         env = dict(os.environ, ORACLE_LIB=so_path)
         r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider",
                             os.path.join(ROOT, "tests", "test_oracle_pins.py"),
-                            os.path.join(ROOT, "tests", "test_oracle_solvers.py")],
+                            os.path.join(ROOT, "tests", "test_oracle_solvers.py"),
+                            os.path.join(ROOT, "tests", "test_oracle_real.py")],
                            env=env, cwd=ROOT, capture_output=True, text=True, timeout=600)
     return name, r.returncode, r.stdout[-300:]
 
