@@ -151,6 +151,29 @@ int sequential_sample(const js_model *m, int batch, const float *noise_dev, int 
 int js_forward_logits(const js_model *m, int batch, const uint8_t *x_dev, float *logits_dev,
                       void *cuda_stream);
 
+/*
+ * Continuous states with logistic conditionals (the paper's MADE: Section 5.3.1, Appendix C.3).  The model is
+ * a masked MLP created with C = 2 (n_lut = 2, the table is not used): the states x_t are real numbers, the
+ * network reads the states themselves (rounded to bf16 in a JS_BF16 model, like any activation) and gives
+ * position t a location m_t (logit 2t) and a log-scale l_t (logit 2t+1) from x_{<t};
+ *     x_t = m_t + exp(l_t) * noise_t,    noise_t = logit(u_t)   (inverse CDF of the logistic law, Appendix A.3)
+ *   noise_dev        fp32 [batch][T], logistic numbers (as for JS_NOISE_LOGISTIC)
+ *   init_dev         fp32 [batch][T] start iterate s^0, or NULL (zeros)
+ *   eps              >= 0: a sample stops at the first iteration whose largest change max_t |x^k_t - x^{k-1}_t|
+ *                    is <= eps (forward-difference rule of Section 2.2.1 in the maximum norm) or at the
+ *                    algorithm's cap; eps = 0 gives the exact feedforward result (Proposition 1), eps > 0
+ *                    trades error for iterations
+ *   out_states_dev   fp32 [batch][T];  out_iters_dev as in jacobi_sample
+ * Modes JS_JACOBI, JS_GAUSS_SEIDEL and JS_GS_JACOBI (JS_JACOBI_GS: JS_ERR_UNSUPPORTED).  CUDA-core kernels.
+ * js_forward_logits_real gives the [batch][T][2] outputs of the network for given states.
+ */
+int jacobi_sample_real(const js_model *m, int batch, const float *noise_dev, const float *init_dev, int mode,
+                       int block, int max_iters, float eps, float *out_states_dev, int32_t *out_iters_dev,
+                       void *cuda_stream);
+int sequential_sample_real(const js_model *m, int batch, const float *noise_dev, float *out_states_dev,
+                           void *cuda_stream);
+int js_forward_logits_real(const js_model *m, int batch, const float *x_dev, float *logits_dev, void *cuda_stream);
+
 typedef enum {
     JS_OPT_FRONTIER_SKIP = 0,  /* 1 (default): skip positions and hidden units already final (proof of Prop. 1) */
     JS_OPT_SEQ_SKIP = 1,       /* how sequential_sample and JS_GAUSS_SEIDEL walk the strict order.  0: a full forward pass per

@@ -71,6 +71,9 @@ def load_library():
     lib.jacobi_sample_host.argtypes = [vp, ip, vp, ip, vp, ip, ip, ip, vp, vp, vp]
     lib.sequential_sample.argtypes = [vp, ip, vp, ip, vp, vp]
     lib.js_forward_logits.argtypes = [vp, ip, vp, vp, vp]
+    lib.jacobi_sample_real.argtypes = [vp, ip, vp, vp, ip, ip, ip, C.c_float, vp, vp, vp]
+    lib.sequential_sample_real.argtypes = [vp, ip, vp, vp, vp]
+    lib.js_forward_logits_real.argtypes = [vp, ip, vp, vp, vp]
     lib.js_set_option.argtypes = [vp, ip, ip]
     lib.js_get_stats.argtypes = [vp, C.POINTER(JsStats)]
     lib.js_get_trace.argtypes = [vp, vp, ip]
@@ -245,6 +248,29 @@ def js_forward_logits(model: Model, x: torch.Tensor, logits: torch.Tensor, strea
     rc = load_library().js_forward_logits(model._h, batch, _dev(x, torch.uint8, "x"),
                                           _dev(logits, torch.float32, "logits"), _stream_ptr(stream))
     return _check(rc, "js_forward_logits")
+
+
+def jacobi_sample_real(model: Model, noise: torch.Tensor, init: Optional[torch.Tensor], mode: int, block: int,
+                       max_iters: int, eps: float, out_states: torch.Tensor,
+                       out_iters: Optional[torch.Tensor] = None, stream=None) -> int:
+    """jacobi_sample_real of the C ABI: continuous states with logistic conditionals, stopping tolerance eps."""
+    rc = load_library().jacobi_sample_real(
+        model._h, out_states.shape[0], _dev(noise, torch.float32, "noise"), _dev(init, torch.float32, "init"), mode,
+        block, max_iters, float(eps), _dev(out_states, torch.float32, "out_states"),
+        _dev(out_iters, torch.int32, "out_iters"), _stream_ptr(stream))
+    return _check(rc, "jacobi_sample_real")
+
+
+def sequential_sample_real(model: Model, noise: torch.Tensor, out_states: torch.Tensor, stream=None) -> int:
+    rc = load_library().sequential_sample_real(model._h, out_states.shape[0], _dev(noise, torch.float32, "noise"),
+                                               _dev(out_states, torch.float32, "out_states"), _stream_ptr(stream))
+    return _check(rc, "sequential_sample_real")
+
+
+def js_forward_logits_real(model: Model, x: torch.Tensor, logits: torch.Tensor, stream=None) -> int:
+    rc = load_library().js_forward_logits_real(model._h, x.shape[0], _dev(x, torch.float32, "x"),
+                                               _dev(logits, torch.float32, "logits"), _stream_ptr(stream))
+    return _check(rc, "js_forward_logits_real")
 
 
 def _noalloc_net(T: int, Cc: int, H: Sequence[int], act: int, W: List[torch.Tensor], b: List[torch.Tensor],

@@ -194,8 +194,9 @@ int prep_args(js_model *m, RunArgs &r, cudaStream_t st)
     r.smp_changed = m->smp_changed;
     r.smp_state = m->smp_state;
     r.x_old = m->x_old;
-    r.frontier_skip = m->opt_frontier_skip;
-    r.seq_skip = m->opt_seq_skip == 1 ? 1 : 0;
+    // with a tolerance eps > 0 an unchanged position is not a final one: no skipping on continuous states
+    r.frontier_skip = r.real ? 0 : m->opt_frontier_skip;
+    r.seq_skip = (!r.real && m->opt_seq_skip == 1) ? 1 : 0;
     r.compact = m->opt_compact;
     r.perm = m->perm;
     r.perm_stride = m->rows;
@@ -560,6 +561,53 @@ int jacobi_sample_host(const js_model *cm, int batch, const float *noise_host, i
     HOST_TRY(cudaStreamSynchronize(st));
 #undef HOST_TRY
     return rc;
+}
+
+// ---- continuous states (logistic conditionals): masked MLPs with C == 2, CUDA-core kernels
+static bool real_model_ok(const js_model *m) { return m && m->kind == 0 && m->made.C == 2; }
+
+int jacobi_sample_real(const js_model *cm, int batch, const float *noise_dev, const float *init_dev, int mode, int block,
+                       int max_iters, float eps, float *out_states_dev, int32_t *out_iters_dev, void *cuda_stream)
+{
+    js_model *m = const_cast<js_model *>(cm);
+    if (!m || !noise_dev || !out_states_dev) return JS_ERR_ARG;
+    if (!real_model_ok(m)) return JS_ERR_UNSUPPORTED;
+    if (batch < 1 || batch > m->max_batch || !(eps >= 0.0f)) return JS_ERR_ARG;
+    if (mode < JS_JACOBI || mode > JS_JACOBI_GS) return JS_ERR_ARG;
+    if (mode == JS_JACOBI_GS) return JS_ERR_UNSUPPORTED;
+    if (mode == JS_GS_JACOBI && (block < 1 || block > m->made.T)) return JS_ERR_ARG;
+    RunArgs r;
+    memset(&r, 0, sizeof r);
+    r.batch = batch; r.noise = noise_dev; r.nk = JS_NOISE_LOGISTIC;
+    r.kmode = mode == JS_JACOBI ? KM_JACOBI : mode == JS_GAUSS_SEIDEL ? KM_SEQ : KM_GS_JACOBI;
+    r.block = block; r.max_iters = max_iters;
+    r.real = 1; r.eps = eps; r.xr = out_states_dev; r.init_r = init_dev; r.out_iters = out_iters_dev;
+    return run_made(m, r, (cudaStream_t)cuda_stream);
+}
+
+int sequential_sample_real(const js_model *cm, int batch, const float *noise_dev, float *out_states_dev, void *cuda_stream)
+{
+    js_model *m = const_cast<js_model *>(cm);
+    if (!m || !noise_dev || !out_states_dev) return JS_ERR_ARG;
+    if (!real_model_ok(m)) return JS_ERR_UNSUPPORTED;
+    if (batch < 1 || batch > m->max_batch) return JS_ERR_ARG;
+    RunArgs r;
+    memset(&r, 0, sizeof r);
+    r.batch = batch; r.noise = noise_dev; r.nk = JS_NOISE_LOGISTIC; r.kmode = KM_SEQ;
+    r.real = 1; r.xr = out_states_dev;
+    return run_made(m, r, (cudaStream_t)cuda_stream);
+}
+
+int js_forward_logits_real(const js_model *cm, int batch, const float *x_dev, float *logits_dev, void *cuda_stream)
+{
+    js_model *m = const_cast<js_model *>(cm);
+    if (!m || !x_dev || !logits_dev) return JS_ERR_ARG;
+    if (!real_model_ok(m)) return JS_ERR_UNSUPPORTED;
+    if (batch < 1 || batch > m->max_batch) return JS_ERR_ARG;
+    RunArgs r;
+    memset(&r, 0, sizeof r);
+    r.batch = batch; r.kmode = KM_FORWARD; r.real = 1; r.xin_r = x_dev; r.logits_out = logits_dev;
+    return run_made(m, r, (cudaStream_t)cuda_stream);
 }
 
 int sequential_sample(const js_model *cm, int batch, const float *noise_dev, int nk, uint8_t *out_samples_dev,

@@ -69,6 +69,12 @@ struct RunArgs {
     int *perm;                // [2][perm_stride]: working row -> sample index, by compaction parity
     int perm_stride;
     int frontier_skip, seq_skip, compact;
+    // continuous states (C == 2: location and log-scale per position): real != 0, states are floats
+    int real;
+    float eps;                // stop when the largest change of a sample's states is <= eps
+    float *xr;                // working iterate = output states [batch][T]
+    const float *init_r;      // start iterate or NULL (zeros)
+    const float *xin_r;       // KM_FORWARD: states to evaluate the network on
     int blk_lo;               // sweeps: first block that is swept (earlier ones are final)
     int hid_lo;               // KM_HIDDEN: hidden units of degree <= hid_lo are final already
     unsigned spin_limit;

@@ -167,6 +167,55 @@ __device__ void sample_phase(const MadeDev &m, const RunArgs &r, const float *z,
     }
 }
 
+// Continuous states: x = start values (or zeros), a[0] = x (rounded like any activation in a bf16 model).
+template <typename T>
+__device__ void init_phase_real(const MadeDev &m, const RunArgs &r, const float *src)
+{
+    const size_t n = (size_t)r.batch * m.T;
+    T *a0 = (T *)m.a[0];
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const float v = src ? src[i] : 0.0f;
+        if (r.xr) r.xr[i] = v;
+        a0[i] = from_f32<T>(v);
+    }
+    if (blockIdx.x == 0) {
+        for (int i = threadIdx.x; i < 2 * r.batch; i += blockDim.x) {
+            r.smp_changed[i] = 0;
+            r.smp_state[i] = 0;
+        }
+        if (threadIdx.x == 0) {
+            r.ctl->agg_any[0] = r.ctl->agg_any[1] = 0;
+            r.ctl->agg_minfirst[0] = r.ctl->agg_minfirst[1] = INT_MAX;
+        }
+    }
+}
+
+// Continuous states with logistic conditionals (Section 5.3.1, Appendix C.3 of arXiv 2002.03629): logit 2t
+// is the location m_t, logit 2t+1 the log-scale l_t, and the position's reserved noise e_t = logit(u_t) gives
+// x_t = m_t + exp(l_t) e_t (inverse CDF of the logistic law).  A position counts as changed when it moved by
+// more than eps, so "no position changed" is the stopping rule  max_t |x^k_t - x^{k-1}_t| <= eps  of
+// Section 2.2.1 in the maximum norm.
+template <typename T>
+__device__ void sample_real_phase(const MadeDev &m, const RunArgs &r, const float *z, int plo, int phi, bool flag,
+                                  int parity)
+{
+    const int T_ = m.T, np = phi - plo;
+    T *a0 = (T *)m.a[0];
+    const size_t n = (size_t)r.batch * np;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int b = (int)(i / np), d = plo + (int)(i % np);
+        // a sample whose stopping test has fired keeps the iterate it stopped at (with eps > 0 a further
+        // update would still move it)
+        if (flag && r.smp_state[b] != 0) continue;
+        const size_t at = (size_t)b * T_ + d;
+        const float xn = fmaf(expf(z[2 * at + 1]), r.noise[at], z[2 * at]);
+        const float xo = r.xr[at];
+        r.xr[at] = xn;
+        a0[at] = from_f32<T>(xn);
+        if (flag && !(fabsf(xn - xo) <= r.eps)) note_change(r, parity, b, d);     // a NaN difference is a change
+    }
+}
+
 template <typename T>
 __device__ bool forward_pass(Smem &s, const MadeDev &m, const RunArgs &r, T *const *acts, float *zout, const Win &w,
                              unsigned &epoch, unsigned long long &issued, unsigned long long &skipped)
@@ -330,7 +379,13 @@ struct GenericEngine {
         for (int l = 0; l <= m.L; ++l) { acts[l] = (T *)m.a[l]; acts_old[l] = (T *)m.a_old[l]; }
     }
     __device__ bool barrier() { return grid_barrier(r.ctl, epoch, r.spin_limit); }
-    __device__ void init(const uint8_t *src) { init_phase<T>(m, r, src); }
+    __device__ void init(const uint8_t *src)
+    {
+        if (r.real)
+            init_phase_real<T>(m, r, r.kmode == KM_FORWARD ? r.xin_r : r.kmode == KM_SEQ ? (const float *)nullptr : r.init_r);
+        else
+            init_phase<T>(m, r, src);
+    }
     __device__ int compact(int) { return 0; }      // the CUDA-core path keeps the batch as it is
     // one forward pass over the window; then either the logits go to zout (teacher forcing) or
     // positions [w.plo, w.phi) are sampled and committed
@@ -338,7 +393,8 @@ struct GenericEngine {
     {
         if (zout) return forward_pass<T>(s, m, r, acts, zout, w, epoch, issued, skipped);
         if (!forward_pass<T>(s, m, r, acts, m.logits, w, epoch, issued, skipped)) return false;
-        sample_phase<T>(m, r, m.logits, w.plo, w.phi, flag, parity);
+        if (r.real) sample_real_phase<T>(m, r, m.logits, w.plo, w.phi, flag, parity);
+        else sample_phase<T>(m, r, m.logits, w.plo, w.phi, flag, parity);
         return barrier();
     }
     // one outer iteration of Algorithm 2

@@ -18,7 +18,9 @@ def declared_symbols():
 def test_header_declares_the_entry_points():
     names = declared_symbols()
     for must in ("jacobi_sample", "sequential_sample", "js_made_create", "js_conv_create", "js_model_destroy",
-                 "js_forward_logits", "js_set_option", "js_get_stats", "js_strerror", "js_last_cuda_error"):
+                 "js_forward_logits", "js_set_option", "js_get_stats", "js_strerror", "js_last_cuda_error",
+                 "jacobi_sample_host", "jacobi_sample_real", "sequential_sample_real", "js_forward_logits_real",
+                 "jacobi_sample_noalloc", "js_get_trace"):
         assert must in names, names
 
 
