@@ -47,7 +47,7 @@ struct SweepDev {
     int WF[JS_MAXL + 1];
     const int *cnt[JS_MAXL + 1];        // cnt[l][d], d = 0..T: units of a[l] with degree <= d (l >= 1)
     int G;                              // positions per group
-    int n_stages, smem_bytes, slots;
+    int n_stages, ring_bytes, smem_bytes, slots;
 };
 
 // Device view of a masked-convolution stack (tensor-core kernel only).

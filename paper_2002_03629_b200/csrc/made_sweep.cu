@@ -41,7 +41,7 @@ constexpr int GMAX = 32;                     // most positions per group
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int W_BYTES = NUP * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + W_BYTES;          // 20 KB, a multiple of 1 KB
-constexpr int MAX_STAGES = 6;
+constexpr int MAX_STAGES = 10;
 constexpr int SMEM_DYN_MAX = 227 * 1024 - 4 * 1024;
 
 struct SwShared {
@@ -101,9 +101,11 @@ struct SweepEngine {
     {
         warp = threadIdx.x >> 5;
         lane = threadIdx.x & 31;
-        uint8_t *p = ring + (size_t)sw.n_stages * STAGE_BYTES;
-        V = reinterpret_cast<float *>(p);
-        p += (size_t)(m.L + 1) * NUP * BM * 4;
+        // The running sums V live in the operand ring's memory: the ring is idle from the moment a group's
+        // prefix sums are complete until the next group's loads start, which is exactly when V is in use
+        // (the threads fence their accesses against the asynchronous proxy before they let the loads go).
+        V = reinterpret_cast<float *>(ring);
+        uint8_t *p = ring + (size_t)sw.ring_bytes;
         X = reinterpret_cast<float *>(p);
         p += (size_t)NUP * BM * 4;
         Wg = reinterpret_cast<float *>(p);
@@ -427,6 +429,8 @@ struct SweepEngine {
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.gdone);
+            } else {
+                fence_proxy_async();          // the next job's loads will overwrite the running sums
             }
             if (tid == 0) trace(6);
             group_no++;
@@ -587,10 +591,13 @@ int js_sweep_prepare(js_model *mo)
     }
     if (G < 1) return 0;
     s.G = G;
-    const int fixed = (L + 1) * NUP * BM * 4 + NUP * BM * 4 + (L + 1) * NUP * NUP * 4 + GMAX * BM * 4;
+    const int v_bytes = (L + 1) * NUP * BM * 4;            // shares the ring's memory
+    const int fixed = NUP * BM * 4 + (L + 1) * NUP * NUP * 4 + GMAX * BM * 4;
     s.n_stages = std::min(MAX_STAGES, (SMEM_DYN_MAX - 1024 - fixed) / STAGE_BYTES);
     if (s.n_stages < 2) return 0;
-    s.smem_bytes = 1024 + s.n_stages * STAGE_BYTES + fixed;
+    s.ring_bytes = std::max(s.n_stages * STAGE_BYTES, (v_bytes + 1023) / 1024 * 1024);
+    if (1024 + s.ring_bytes + fixed > SMEM_DYN_MAX) return 0;
+    s.smem_bytes = 1024 + s.ring_bytes + fixed;
     int dev = 0, sms = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
