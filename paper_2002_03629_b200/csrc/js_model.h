@@ -42,7 +42,7 @@ struct TcDev {
 struct SweepDev {
     const CUtensorMap *tmAold;          // [L+1] activations a[l] of the previous iterate, box 64 x 128 (= TcDev::tmA)
     const CUtensorMap *tmF;             // [L+1] the jobs' buffers F[l], 3-D {column, row, slot}, box 64 x 128 x 1
-    const CUtensorMap *tmW16;           // [L+1] masked weights W[l], box 64 x 16
+    const CUtensorMap *tmW16;           // [2][L+1] masked weights W[l]: box 64 x 16 rows, then box 64 x 32 rows
     __nv_bfloat16 *F[JS_MAXL + 1];      // [slot][128 rows][WF[l]]: a job's fresh activations of a[l]
     int WF[JS_MAXL + 1];
     const int *cnt[JS_MAXL + 1];        // cnt[l][d], d = 0..T: units of a[l] with degree <= d (l >= 1)

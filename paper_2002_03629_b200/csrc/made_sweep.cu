@@ -177,9 +177,9 @@ struct SweepEngine {
                         tma_load_2d(smem_u32(stage_a(stage)), sw.tmAold + l, &sh.full[stage], kb * BK, rt * BM);
                     else
                         tma_load_3d(smem_u32(stage_a(stage)), sw.tmF + l, &sh.full[stage], (kb - kb_old[l]) * BK, 0, slot);
-                    for (int i = 0; i < g.npad / 16; ++i)
-                        tma_load_2d(smem_u32(stage_b(stage)) + i * 16 * BK * 2, sw.tmW16 + l, &sh.full[stage], kb * BK,
-                                    g.u0 + i * 16);
+                    // one box of 16 or of 32 weight rows (a load per 16 rows cost a fifth of the K loop)
+                    tma_load_2d(smem_u32(stage_b(stage)), sw.tmW16 + (g.npad == 32 ? m.L + 1 : 0) + l, &sh.full[stage],
+                                kb * BK, g.u0);
                     advance_stage();
                 }
             }
@@ -604,7 +604,7 @@ int js_sweep_prepare(js_model *mo)
     if (sms < 1) return 0;
     s.slots = sms;
     auto fail = [&]() { cudaGetLastError(); return JS_ERR_CUDA; };
-    std::vector<CUtensorMap> mapsF(L + 1), mapsW(L + 1);
+    std::vector<CUtensorMap> mapsF(L + 1), mapsW(2 * (L + 1));       // weights: boxes of 16 rows, then of 32 rows
     for (int l = 0; l <= L; ++l) {
         if (l >= 1) {
             void *p = nullptr;
@@ -628,20 +628,20 @@ int js_sweep_prepare(js_model *mo)
             const cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BM, 1};
             if (!sweep_encode(&mapsF[l], f, 3, dims, strides, box)) return 0;
         }
-        {
+        for (int big = 0; big < 2; ++big) {
             const cuuint64_t dims[2] = {(cuuint64_t)v.n[l], (cuuint64_t)v.n[l + 1]};
             const cuuint64_t strides[1] = {(cuuint64_t)v.n[l] * 2};
-            const cuuint32_t box[2] = {(cuuint32_t)BK, 16};
-            if (!sweep_encode(&mapsW[l], v.W[l], 2, dims, strides, box)) return 0;
+            const cuuint32_t box[2] = {(cuuint32_t)BK, big ? 32u : 16u};
+            if (!sweep_encode(&mapsW[big * (L + 1) + l], v.W[l], 2, dims, strides, box)) return 0;
         }
     }
     void *pf = nullptr, *pw = nullptr;
     if (cudaMalloc(&pf, (L + 1) * sizeof(CUtensorMap)) != cudaSuccess) return fail();
     mo->allocs.push_back(pf);
-    if (cudaMalloc(&pw, (L + 1) * sizeof(CUtensorMap)) != cudaSuccess) return fail();
+    if (cudaMalloc(&pw, 2 * (L + 1) * sizeof(CUtensorMap)) != cudaSuccess) return fail();
     mo->allocs.push_back(pw);
     if (cudaMemcpy(pf, mapsF.data(), (L + 1) * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess) return fail();
-    if (cudaMemcpy(pw, mapsW.data(), (L + 1) * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess) return fail();
+    if (cudaMemcpy(pw, mapsW.data(), 2 * (L + 1) * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess) return fail();
     s.tmF = (const CUtensorMap *)pf;
     s.tmW16 = (const CUtensorMap *)pw;
     s.tmAold = mo->tc.tmA;
