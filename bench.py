@@ -173,6 +173,14 @@ def make_inputs(cfg):
     return W, b, si.made_lut(cfg), si.draw_noise(cfg)
 
 
+def config_of(cfg, mode, block, world):
+    """The `config` object of the JSON line: the same in both arms, so that the two lines can be paired."""
+    return {"workload": cfg.name, "mode": mode, "block": block, "batch": cfg.batch, "T": cfg.D, "C": cfg.C,
+            "hidden": list(cfg.H) if cfg.kind == "made" else [cfg.ch] * cfg.layers,
+            "parallelism": f"replicas x{world}",
+            "l2": "256 MB written between timed GPU steps (L2 flush)"}
+
+
 # -------------------------------------------------------------- reference arm
 def oracle_sample_time(cfg, W, b, lut, noise, mode, block, n_samples, threads):
     """Oracle wall time for n_samples of the workload in the given mode (as it stands, untuned)."""
@@ -215,8 +223,7 @@ def run_reference(args, cfg):
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": cfg.name, "mode": args.mode, "block": args.block, "batch": cfg.batch,
-                       "sample": f"{n} of {cfg.batch} samples per step"},
+            "config": config_of(cfg, args.mode, args.block, args.gpus),
             "iters_per_sample_mean": float(np.mean(its)),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": min(cores, n), "kind": "oracle",
                              "sample": f"{n} samples x {args.steps} steps, {args.mode}"},
@@ -448,10 +455,7 @@ def run_ours(args, cfg):
     line = {"metric": METRIC, "value": rec["samples_per_s"], "unit": UNIT, "n_gpus": world, "steps": steps,
             "warmup": max(args.warmup, 3), "ms_per_step": rec["ms_per_call"], "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": dtype, "data": "synthetic",
-            "config": {"workload": cfg.name, "mode": args.mode, "block": args.block, "batch": cfg.batch, "T": cfg.D,
-                       "C": cfg.C, "hidden": list(cfg.H) if cfg.kind == "made" else [cfg.ch] * cfg.layers,
-                       "parallelism": f"replicas x{world}",
-                       "l2": "256 MB written between timed steps (L2 flush)"},
+            "config": config_of(cfg, args.mode, args.block, world),
             "iters_per_sample": rec["iters_per_sample"],
             "kernel_path": rec["kernel_path"],
             "tiles": rec["tiles"],
