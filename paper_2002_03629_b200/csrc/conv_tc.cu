@@ -22,7 +22,7 @@
 namespace {
 
 constexpr int BM = TC_BM, BK = TC_BK;
-constexpr int NTH = 192;
+constexpr int NTH = 320;          // warp 0 loads, warp 1 MMA, warps 2-9 epilogue: two per tensor-memory lane quadrant
 constexpr int ACC_COLS = 256;
 constexpr int A_BYTES = BM * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + 256 * BK * 2;   // A tile + up to 256 weight rows
@@ -46,8 +46,11 @@ struct ConvShared {
     uint64_t full[N_STAGES], empty[N_STAGES], tfull[2], tempty[2];
     uint32_t tmem_base;
     float bias_s[4][256];
+    float xbest[2][4][32];    // head: the upper class half's best score and class, by tile parity and quadrant
+    int xbi[2][4][32];
     float lut_s[256];         // input encoding table
     int img[MAX_IMAGES];      // images still iterating
+    unsigned char keep[MAX_IMAGES];
     int n_img;
 };
 
@@ -127,12 +130,15 @@ struct ConvEngine {
     __device__ int compact(int parity)
     {
         __syncthreads();
+        // the flags are fetched by as many threads as there are images (one thread reading them one after
+        // the other paid an L2 round trip per image, 7 us per pass on a batch of 16), then one thread packs
+        for (int i = threadIdx.x; i < sh.n_img; i += blockDim.x)
+            sh.keep[i] = ld_volatile_i32(&r.smp_changed[parity * r.batch + sh.img[i]]) != 0 ? 1 : 0;
+        __syncthreads();
         if (threadIdx.x == 0) {
             int k = 0;
-            for (int i = 0; i < sh.n_img; ++i) {
-                const int b = sh.img[i];
-                if (ld_volatile_i32(&r.smp_changed[parity * r.batch + b]) != 0) sh.img[k++] = b;
-            }
+            for (int i = 0; i < sh.n_img; ++i)
+                if (sh.keep[i]) sh.img[k++] = sh.img[i];
             sh.n_img = k;
             if (blockIdx.x == 0) { r.ctl->compactions += 1; r.ctl->live = k; }
         }
@@ -340,12 +346,25 @@ struct ConvEngine {
         const bool head = (l == m.n_conv);
         const int per = head ? m.in_ch : 1;
         const int q = warp & 3;
+        // Two warps share a quadrant (a warp reaches only the tensor-memory lanes of its own quadrant).  The
+        // second one takes the upper 128 classes of a 256-way head tile: the argmax is bound by instruction
+        // issue, one warp per scheduler was not enough; elsewhere it only hands the accumulator back.
+        const int half = (warp - 2) >> 2;
+        int tile_par = 0;
         bool any_changed = false;
         int first = INT_MAX;
         for (int id = blockIdx.x; id < ntiles && !dead; id += gridDim.x) {
             int n, yt, c;
             locate(id, nyl, yt_lo, per, n, yt, c);
             const int y0 = yt * m.R;
+            const bool split_head = head && kind == EPI_CAT && r.nk == JS_NOISE_GUMBEL;
+            if (half == 1 && !(head && (split_head || kind == EPI_LOGITS))) {
+                if (!mbar_wait(&sh.tfull[acc], aphase, r.ctl)) { dead = true; break; }
+                tc_fence_after();
+                release_acc();
+                advance_acc();
+                continue;
+            }
             if (!head) {
                 float *bs = sh.bias_s[warp - 2];
                 __syncwarp();
@@ -376,7 +395,7 @@ struct ConvEngine {
                 if (kind == EPI_CAT && r.nk == JS_NOISE_UNIFORM_CAT) {
                     bi = head_icdf(tbase, bias, commit ? __ldg(r.noise + at) : 0.5f);
                 } else
-                for (int c0 = 0; c0 < 256; c0 += 32) {
+                for (int c0 = half * 128; c0 < half * 128 + 128; c0 += 32) {
                     float v[32];
                     __syncwarp();
                     tmem_ld32(tbase + (uint32_t)c0, v);
@@ -400,6 +419,20 @@ struct ConvEngine {
                     }
                 }
                 release_acc();        // the accumulator has been read: the next tile's MMAs may have it
+                if (split_head) {
+                    // the two halves meet: the upper half's result wins only if strictly larger (lowest index on ties)
+                    if (half == 1) {
+                        sh.xbest[tile_par][q][lane] = best;
+                        sh.xbi[tile_par][q][lane] = bi;
+                    }
+                    asm volatile("bar.sync %0, 64;" ::"r"(1 + q) : "memory");
+                    if (half == 0) {
+                        const float b1 = sh.xbest[tile_par][q][lane];
+                        if (b1 > best) { best = b1; bi = sh.xbi[tile_par][q][lane]; }
+                    }
+                    tile_par ^= 1;
+                }
+                if (half == 1) { advance_acc(); continue; }
                 bool ch = false;
                 if (commit && xold != bi) {
                     r.x[at] = (uint8_t)bi;
@@ -545,7 +578,7 @@ conv_tc_kernel(const __grid_constant__ ConvDev m, const __grid_constant__ RunArg
     const int warp = threadIdx.x >> 5;
     if (threadIdx.x == 0) {
         for (int s = 0; s < N_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 8); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
     }
