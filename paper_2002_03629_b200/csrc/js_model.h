@@ -42,7 +42,9 @@ struct TcDev {
 struct SweepDev {
     const CUtensorMap *tmAold;          // [L+1] activations a[l] of the previous iterate, box 64 x 128 (= TcDev::tmA)
     const CUtensorMap *tmF;             // [L+1] the jobs' buffers F[l], 3-D {column, row, slot}, box 64 x 128 x 1
-    const CUtensorMap *tmW16;           // [2][L+1] masked weights W[l]: box 64 x 16 rows, then box 64 x 32 rows
+    const CUtensorMap *tmW16;           // [3][L+1] masked weights W[l]: boxes of 64 x 16, 64 x 32 and 64 x 64 (columns x rows)
+    float *S;                           // [slot][L+1][nbs][128 rows] fp32: base sums of a job's next groups
+    int nbs;
     __nv_bfloat16 *F[JS_MAXL + 1];      // [slot][128 rows][WF[l]]: a job's fresh activations of a[l]
     int WF[JS_MAXL + 1];
     const int *cnt[JS_MAXL + 1];        // cnt[l][d], d = 0..T: units of a[l] with degree <= d (l >= 1)

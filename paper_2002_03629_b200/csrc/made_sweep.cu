@@ -39,13 +39,17 @@ constexpr int NTH = 192;
 constexpr int NUP = 32;                      // most units of one layer inside a group
 constexpr int GMAX = 32;                     // most positions per group
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int W_BYTES = NUP * BK * 2;
-constexpr int STAGE_BYTES = A_BYTES + W_BYTES;          // 20 KB, a multiple of 1 KB
+constexpr int NB = 64;                       // units per chunk of a base GEMM
+constexpr int GPB = 4;                       // groups per base: a base GEMM serves the next GPB groups
+constexpr int W_BYTES = NB * BK * 2;
+constexpr int STAGE_BYTES = A_BYTES + W_BYTES;          // 24 KB, a multiple of 1 KB
+constexpr int BASE_COL = 320;                // tensor-memory columns of the two base accumulators (64 each)
 constexpr int MAX_STAGES = 10;
 constexpr int SMEM_DYN_MAX = 227 * 1024 - 4 * 1024;
 
 struct SwShared {
-    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tfull, tempty, gdone;
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], tfull, tempty, gdone, bfull[2], bempty[2];
+    int kbs[JS_MAXL + 1], ub0[JS_MAXL + 1];  // current base: its K blocks per layer (0: none), its first unit
     uint32_t tmem_base;
     int stop;
     float lut_s[2];
@@ -56,6 +60,7 @@ struct SwShared {
 };
 
 struct Geo { int kin0, kb_n, nin, u0, nu, npad; };
+struct Base { int kbs, ub0, nb; };           // K blocks [0, kbs), units [ub0, ub0 + nb)
 
 // shared-memory accesses by 32-bit shared address: the position loop runs on one warp per scheduler, and
 // a generic load (which is what a pointer kept in a structure compiles to) waits much longer than ld.shared
@@ -92,6 +97,8 @@ struct SweepEngine {
     int stage = 0;
     uint32_t spar = 0;
     uint32_t tf_par = 0, te_par = 0, gd_par = 0;
+    int bbuf = 0;                  // base accumulator in turn; bit b of bb_par: parity of its next use
+    uint32_t bb_par = 0;
     bool dead = false;
     uint32_t tmem_base = 0;
     unsigned long long mma_flops = 0;
@@ -144,6 +151,26 @@ struct SweepEngine {
         return g;
     }
 
+    // Base of the GPB groups that start at position s0 (block ends at b): per layer, the sums over all FULL
+    // K blocks below the first group's prefix boundary, for every unit those groups will evaluate.  The
+    // groups' own GEMMs then run only over the K blocks from there on.
+    __device__ Base base_of(int l, int s0, int b) const
+    {
+        const int sE = min(s0 + GPB * sw.G, b), hiS = min(sE, b - 1);
+        Base g;
+        g.kbs = cnt(l, s0) / BK;
+        if (l < m.L) {
+            g.ub0 = cnt(l + 1, s0);
+            g.nb = cnt(l + 1, hiS) - g.ub0;
+        } else {
+            g.ub0 = s0;
+            g.nb = sE - s0;
+        }
+        if (g.nb <= 0) g.kbs = 0;
+        return g;
+    }
+    __device__ int base_start(int a, int t0) const { return a + ((t0 - a) / (GPB * sw.G)) * (GPB * sw.G); }
+
     __device__ uint8_t *stage_a(int s) const { return ring + (size_t)s * STAGE_BYTES; }
     __device__ uint8_t *stage_b(int s) const { return ring + (size_t)s * STAGE_BYTES + A_BYTES; }
     __device__ uint32_t stage_parity() const { return (spar >> stage) & 1u; }
@@ -165,12 +192,34 @@ struct SweepEngine {
             gd_par ^= 1u;
             fence_proxy_async();
             trace(0);
+            const int s0 = base_start(a, t0);
+            if (t0 == s0) {
+                // the base GEMMs of the next GPB groups: 64 units at a time over the full K blocks of the prefix
+                for (int l = 0; l <= m.L && !dead; ++l) {
+                    const Base bs = base_of(l, s0, b);
+                    for (int c = 0; c * NB < bs.nb && bs.kbs > 0 && !dead; ++c) {
+                        mma_flops += 2ull * BM * BK * NB * (unsigned long long)bs.kbs;
+                        for (int kb = 0; kb < bs.kbs; ++kb) {
+                            if (!mbar_wait(&sh.empty[stage], stage_parity() ^ 1u, r.ctl)) { dead = true; break; }
+                            mbar_expect_tx(&sh.full[stage], A_BYTES + NB * BK * 2);
+                            if (kb < kb_old[l])
+                                tma_load_2d(smem_u32(stage_a(stage)), sw.tmAold + l, &sh.full[stage], kb * BK, rt * BM);
+                            else
+                                tma_load_3d(smem_u32(stage_a(stage)), sw.tmF + l, &sh.full[stage], (kb - kb_old[l]) * BK, 0, slot);
+                            tma_load_2d(smem_u32(stage_b(stage)), sw.tmW16 + 2 * (m.L + 1) + l, &sh.full[stage], kb * BK,
+                                        bs.ub0 + c * NB);
+                            advance_stage();
+                        }
+                    }
+                }
+            }
             for (int l = 0; l <= m.L && !dead; ++l) {
                 const Geo g = geo(l, t0, t1, hi);
                 if (g.nu == 0) continue;
                 const uint32_t bytes = A_BYTES + (uint32_t)g.npad * BK * 2;
-                mma_flops += 2ull * BM * BK * (unsigned long long)g.npad * (unsigned long long)g.kb_n;
-                for (int kb = 0; kb < g.kb_n; ++kb) {
+                const int kbs = base_of(l, s0, b).kbs;
+                mma_flops += 2ull * BM * BK * (unsigned long long)g.npad * (unsigned long long)(g.kb_n - kbs);
+                for (int kb = kbs; kb < g.kb_n; ++kb) {
                     if (!mbar_wait(&sh.empty[stage], stage_parity() ^ 1u, r.ctl)) { dead = true; break; }
                     mbar_expect_tx(&sh.full[stage], bytes);
                     if (kb < kb_old[l])
@@ -196,12 +245,43 @@ struct SweepEngine {
             te_par ^= 1u;
             tc_fence_after();
             bool any = false;
+            const int s0 = base_start(a, t0);
+            if (t0 == s0) {
+                const uint32_t idesc64 = instr_desc_bf16(NB);
+                for (int l = 0; l <= m.L && !dead; ++l) {
+                    const Base bs = base_of(l, s0, b);
+                    for (int c = 0; c * NB < bs.nb && bs.kbs > 0 && !dead; ++c) {
+                        // the epilogue has copied this accumulator's previous chunk away
+                        if (!mbar_wait(&sh.bempty[bbuf], ((bb_par >> bbuf) & 1u) ^ 1u, r.ctl)) { dead = true; break; }
+                        tc_fence_after();
+                        const uint32_t d_base = tmem_base + (uint32_t)(BASE_COL + bbuf * NB);
+                        for (int kb = 0; kb < bs.kbs; ++kb) {
+                            if (!mbar_wait(&sh.full[stage], stage_parity(), r.ctl)) { dead = true; break; }
+                            tc_fence_after();
+                            const uint64_t adesc = smem_desc_sw128(smem_u32(stage_a(stage)));
+                            const uint64_t bdesc = smem_desc_sw128(smem_u32(stage_b(stage)));
+#pragma unroll
+                            for (int k = 0; k < BK / 16; ++k)
+                                umma_bf16(d_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc64,
+                                          (kb > 0 || k > 0) ? 1u : 0u);
+                            umma_commit(&sh.empty[stage]);
+                            advance_stage();
+                        }
+                        if (dead) break;
+                        umma_commit(&sh.bfull[bbuf]);
+                        bb_par ^= 1u << bbuf;
+                        bbuf ^= 1;
+                    }
+                }
+                if (dead) break;
+            }
             for (int l = 0; l <= m.L && !dead; ++l) {
                 const Geo g = geo(l, t0, t1, hi);
                 if (g.nu == 0) continue;
                 const uint32_t idesc = instr_desc_bf16(g.npad);
                 const uint32_t d_tmem = tmem_base + (uint32_t)(l * NUP);
-                for (int kb = 0; kb < g.kb_n; ++kb) {
+                const int kbs = base_of(l, s0, b).kbs;
+                for (int kb = kbs; kb < g.kb_n; ++kb) {
                     if (!mbar_wait(&sh.full[stage], stage_parity(), r.ctl)) { dead = true; break; }
                     tc_fence_after();
                     const uint64_t adesc = smem_desc_sw128(smem_u32(stage_a(stage)));
@@ -209,7 +289,7 @@ struct SweepEngine {
 #pragma unroll
                     for (int k = 0; k < BK / 16; ++k)
                         umma_bf16(d_tmem, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc,
-                                  (kb > 0 || k > 0) ? 1u : 0u);
+                                  (kb > kbs || k > 0) ? 1u : 0u);
                     umma_commit(&sh.empty[stage]);
                     advance_stage();
                     any = true;
@@ -316,9 +396,12 @@ struct SweepEngine {
             const int t1 = min(t0 + sw.G, b), hi = min(t1, b - 1), ng = t1 - t0;
             // ---- geometry, small tables, the weights between the group's units, noise (while the GEMMs run)
             ep_sync();                                   // everybody is done with the previous group's tables
+            const int s0 = base_start(a, t0);
             if (tid <= L) {
                 const Geo g = geo(tid, t0, t1, hi);
                 sh.kin0[tid] = g.kin0; sh.nin[tid] = g.nin; sh.u0[tid] = g.u0; sh.nu[tid] = g.nu; sh.kb_n[tid] = g.kb_n;
+                const Base bs = base_of(tid, s0, b);
+                sh.kbs[tid] = bs.kbs; sh.ub0[tid] = bs.ub0;
             }
             for (int i = tid; i < (L + 1) * (GMAX + 2); i += 128) {
                 const int l = i / (GMAX + 2), k = i % (GMAX + 2);
@@ -366,6 +449,31 @@ struct SweepEngine {
             }
             ep_sync();
             if (tid == 0) trace(2);
+            // ---- a new base: its sums go from tensor memory to this job's part of S, chunk by chunk, as the
+            // MMAs deliver them; thread = sample row writes, and later reads, only its own row
+            if (t0 == s0) {
+                for (int l = 0; l <= L && !dead; ++l) {
+                    const Base bs = base_of(l, s0, b);
+                    float *Sl = sw.S + (((size_t)slot * (L + 1) + l) * sw.nbs) * BM + row;
+                    for (int c = 0; c * NB < bs.nb && bs.kbs > 0; ++c) {
+                        if (!mbar_wait(&sh.bfull[bbuf], (bb_par >> bbuf) & 1u, r.ctl)) { dead = true; break; }
+                        tc_fence_after();
+#pragma unroll
+                        for (int h = 0; h < NB; h += 32) {
+                            float v[32];
+                            tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(BASE_COL + bbuf * NB + h), v);
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) Sl[(size_t)(c * NB + h + i) * BM] = v[i];
+                        }
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&sh.bempty[bbuf]);
+                        bb_par ^= 1u << bbuf;
+                        bbuf ^= 1;
+                    }
+                }
+                if (dead) break;
+            }
             // ---- prefix sums out of tensor memory
             if (!mbar_wait(&sh.tfull, tf_par, r.ctl)) { dead = true; break; }
             tf_par ^= 1u;
@@ -373,11 +481,21 @@ struct SweepEngine {
             if (tid == 0) trace(3);
             for (int l = 0; l <= L; ++l) {
                 float v[32];
-                if (sh.nu[l] > 0 && sh.kb_n[l] > 0) {
+                if (sh.nu[l] > 0 && sh.kb_n[l] > sh.kbs[l]) {
                     tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(l * NUP), v);
                 } else {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = 0.0f;
+                }
+                if (sh.kbs[l] > 0 && sh.nu[l] > 0) {
+                    // base + the group's own K blocks (in that order, always)
+                    const float *Sl = sw.S + (((size_t)slot * (L + 1) + l) * sw.nbs + (sh.u0[l] - sh.ub0[l])) * BM + row;
+                    const int nuv = sh.nu[l];
+                    float sv[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) sv[i] = i < nuv ? __ldcg(Sl + (size_t)i * BM) : 0.0f;
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = sv[i] + v[i];
                 }
                 // running pre-activation of every unit of the group: prefix sum + bias; the group's own
                 // contributions are added below, each as soon as its source exists
@@ -450,6 +568,7 @@ made_sweep_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ Swe
         mbar_init(&sh.tfull, 1);
         mbar_init(&sh.tempty, 4);
         mbar_init(&sh.gdone, 4);
+        for (int i = 0; i < 2; ++i) { mbar_init(&sh.bfull[i], 1); mbar_init(&sh.bempty[i], 4); }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_proxy_async();
         sh.lut_s[0] = m.lut[0];
@@ -567,6 +686,7 @@ int js_sweep_prepare(js_model *mo)
     const MadeDev &v = mo->made;
     SweepDev &s = mo->sweep;
     if (!mo->tc_ok || v.C != 1 || v.prec != JS_BF16 || !sweep_encode_fn()) return 0;
+    if ((v.L + 1) * NUP > BASE_COL) return 0;              // the groups' accumulators end where the base's begin
     const int L = v.L, T = v.T;
     // prefix counts; the group size is the largest one that keeps every layer's units of a group within NUP
     std::vector<std::vector<int>> cnt(L + 1);
@@ -604,7 +724,7 @@ int js_sweep_prepare(js_model *mo)
     if (sms < 1) return 0;
     s.slots = sms;
     auto fail = [&]() { cudaGetLastError(); return JS_ERR_CUDA; };
-    std::vector<CUtensorMap> mapsF(L + 1), mapsW(2 * (L + 1));       // weights: boxes of 16 rows, then of 32 rows
+    std::vector<CUtensorMap> mapsF(L + 1), mapsW(3 * (L + 1));       // weights: boxes of 16, of 32 and of 64 rows
     for (int l = 0; l <= L; ++l) {
         if (l >= 1) {
             void *p = nullptr;
@@ -628,23 +748,36 @@ int js_sweep_prepare(js_model *mo)
             const cuuint32_t box[3] = {(cuuint32_t)BK, (cuuint32_t)BM, 1};
             if (!sweep_encode(&mapsF[l], f, 3, dims, strides, box)) return 0;
         }
-        for (int big = 0; big < 2; ++big) {
+        for (int big = 0; big < 3; ++big) {
             const cuuint64_t dims[2] = {(cuuint64_t)v.n[l], (cuuint64_t)v.n[l + 1]};
             const cuuint64_t strides[1] = {(cuuint64_t)v.n[l] * 2};
-            const cuuint32_t box[2] = {(cuuint32_t)BK, big ? 32u : 16u};
+            const cuuint32_t box[2] = {(cuuint32_t)BK, 16u << big};
             if (!sweep_encode(&mapsW[big * (L + 1) + l], v.W[l], 2, dims, strides, box)) return 0;
         }
     }
     void *pf = nullptr, *pw = nullptr;
     if (cudaMalloc(&pf, (L + 1) * sizeof(CUtensorMap)) != cudaSuccess) return fail();
     mo->allocs.push_back(pf);
-    if (cudaMalloc(&pw, 2 * (L + 1) * sizeof(CUtensorMap)) != cudaSuccess) return fail();
+    if (cudaMalloc(&pw, 3 * (L + 1) * sizeof(CUtensorMap)) != cudaSuccess) return fail();
     mo->allocs.push_back(pw);
     if (cudaMemcpy(pf, mapsF.data(), (L + 1) * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess) return fail();
-    if (cudaMemcpy(pw, mapsW.data(), 2 * (L + 1) * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess) return fail();
+    if (cudaMemcpy(pw, mapsW.data(), 3 * (L + 1) * sizeof(CUtensorMap), cudaMemcpyHostToDevice) != cudaSuccess) return fail();
     s.tmF = (const CUtensorMap *)pf;
     s.tmW16 = (const CUtensorMap *)pw;
     s.tmAold = mo->tc.tmA;
+    {
+        // base sums: per slot and layer, room for the units of GPB groups (rounded up to whole chunks)
+        int nbs = NB;
+        for (int l = 1; l <= L; ++l)
+            for (int d = 0; d < T; ++d) nbs = std::max(nbs, cnt[l][std::min(d + GPB * G, T)] - cnt[l][d]);
+        nbs = std::max(nbs, GPB * G);
+        s.nbs = (nbs + NB - 1) / NB * NB;
+        void *p = nullptr;
+        const size_t bytes = (size_t)s.slots * (L + 1) * s.nbs * BM * sizeof(float);
+        if (cudaMalloc(&p, bytes) != cudaSuccess) return fail();
+        mo->allocs.push_back(p);
+        s.S = (float *)p;
+    }
     {
         void *p = nullptr;
         if (cudaMalloc(&p, 2 * (size_t)mo->rows * sizeof(int)) != cudaSuccess) return fail();
