@@ -39,11 +39,11 @@ constexpr int NTH = 192;
 constexpr int NUP = 32;                      // most units of one layer inside a group
 constexpr int GMAX = 32;                     // most positions per group
 constexpr int A_BYTES = BM * BK * 2;
-constexpr int NB = 64;                       // units per chunk of a base GEMM
-constexpr int GPB = 4;                       // groups per base: a base GEMM serves the next GPB groups
+constexpr int NB = 128;                      // units per chunk of a base GEMM
+constexpr int GPB = 8;                       // groups per base: a base GEMM serves the next GPB groups
 constexpr int W_BYTES = NB * BK * 2;
-constexpr int STAGE_BYTES = A_BYTES + W_BYTES;          // 24 KB, a multiple of 1 KB
-constexpr int BASE_COL = 320;                // tensor-memory columns of the two base accumulators (64 each)
+constexpr int STAGE_BYTES = A_BYTES + W_BYTES;          // 32 KB, a multiple of 1 KB
+constexpr int BASE_COL = 256;                // tensor-memory columns of the two base accumulators (NB each)
 constexpr int MAX_STAGES = 10;
 constexpr int SMEM_DYN_MAX = 227 * 1024 - 4 * 1024;
 
@@ -194,7 +194,7 @@ struct SweepEngine {
             trace(0);
             const int s0 = base_start(a, t0);
             if (t0 == s0) {
-                // the base GEMMs of the next GPB groups: 64 units at a time over the full K blocks of the prefix
+                // the base GEMMs of the next GPB groups: NB units at a time over the full K blocks of the prefix
                 for (int l = 0; l <= m.L && !dead; ++l) {
                     const Base bs = base_of(l, s0, b);
                     for (int c = 0; c * NB < bs.nb && bs.kbs > 0 && !dead; ++c) {
@@ -247,7 +247,7 @@ struct SweepEngine {
             bool any = false;
             const int s0 = base_start(a, t0);
             if (t0 == s0) {
-                const uint32_t idesc64 = instr_desc_bf16(NB);
+                const uint32_t idescb = instr_desc_bf16(NB);
                 for (int l = 0; l <= m.L && !dead; ++l) {
                     const Base bs = base_of(l, s0, b);
                     for (int c = 0; c * NB < bs.nb && bs.kbs > 0 && !dead; ++c) {
@@ -262,7 +262,7 @@ struct SweepEngine {
                             const uint64_t bdesc = smem_desc_sw128(smem_u32(stage_b(stage)));
 #pragma unroll
                             for (int k = 0; k < BK / 16; ++k)
-                                umma_bf16(d_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idesc64,
+                                umma_bf16(d_base, adesc + (uint64_t)(2 * k), bdesc + (uint64_t)(2 * k), idescb,
                                           (kb > 0 || k > 0) ? 1u : 0u);
                             umma_commit(&sh.empty[stage]);
                             advance_stage();
@@ -313,8 +313,11 @@ struct SweepEngine {
 
     // source k of a[l] has the value `val`: add its contribution to the running sums of the group's units
     // of a[l+1] (masked weights are zero where the target may not read the source)
-    __device__ void scatter(int l, int k, float val, int row)
+    // Targets below jmin cannot read this source (their degree is lower, their masked weight zero): their
+    // 16-byte chunks are left alone, which halves the shared-memory traffic that bounds the position loop.
+    __device__ void scatter(int l, int k, float val, int row, int jmin)
     {
+        const int c0 = jmin >> 2;
         // the row's 32 running sums as eight 16-byte accesses, all loads before all stores: one warp per
         // scheduler cannot hide the latency of a load that waits behind a store it might alias
         const uint32_t w4 = smem_u32(Wg) + 4u * (uint32_t)((l * NUP + k) * NUP);
@@ -322,18 +325,22 @@ struct SweepEngine {
         const int sw7 = row & 7;
         float4 w[NUP / 4], x[NUP / 4];
 #pragma unroll
-        for (int c = 0; c < NUP / 4; ++c) w[c] = lds_f4(w4 + 16u * c);
+        for (int c = 0; c < NUP / 4; ++c)
+            if (c >= c0) w[c] = lds_f4(w4 + 16u * c);
 #pragma unroll
-        for (int c = 0; c < NUP / 4; ++c) x[c] = lds_f4(v4 + 16u * (uint32_t)(c ^ sw7));
+        for (int c = 0; c < NUP / 4; ++c)
+            if (c >= c0) x[c] = lds_f4(v4 + 16u * (uint32_t)(c ^ sw7));
 #pragma unroll
         for (int c = 0; c < NUP / 4; ++c) {
+            if (c < c0) continue;
             x[c].x = fmaf(w[c].x, val, x[c].x);
             x[c].y = fmaf(w[c].y, val, x[c].y);
             x[c].z = fmaf(w[c].z, val, x[c].z);
             x[c].w = fmaf(w[c].w, val, x[c].w);
         }
 #pragma unroll
-        for (int c = 0; c < NUP / 4; ++c) sts_f4(v4 + 16u * (uint32_t)(c ^ sw7), x[c]);
+        for (int c = 0; c < NUP / 4; ++c)
+            if (c >= c0) sts_f4(v4 + 16u * (uint32_t)(c ^ sw7), x[c]);
     }
 
     // n consecutive values (unit j = 0..n-1 of layer slot l, or the group's encodings when l < 0) of this
@@ -408,42 +415,52 @@ struct SweepEngine {
                 if (l >= 1) sh.cs[l][k] = cnt(l, min(t0 + k, m.T));
             }
             ep_sync();
-            for (int l = 0; l <= L; ++l) {
-                const int nu = sh.nu[l], nin = sh.nin[l], u0 = sh.u0[l], kin0 = sh.kin0[l];
-                const __nv_bfloat16 *Wl = (const __nv_bfloat16 *)m.W[l];
-                const int K = m.n[l];
-                // all loads of a thread first, then its stores: the compiler may not move a load
-                // across a store it cannot tell apart, and eight dependent round trips per layer
-                // would cost more than the group's GEMMs
-                __nv_bfloat16 wv[NUP * NUP / 128];
+            {
+                // Every global load of the thread first, the stores to shared memory after them: the compiler
+                // may not move a load across a store it cannot tell apart, and one round trip per layer and
+                // per table would cost more than the group's GEMMs.
+                constexpr int LB = 3;            // layers per round trip
+                for (int l0 = 0; l0 <= L; l0 += LB) {
+                    __nv_bfloat16 wv[LB][NUP * NUP / 128];
+                    float bv[LB];
 #pragma unroll
-                for (int e = 0; e < NUP * NUP / 128; ++e) {
-                    const int i = tid + e * 128, j = i / NUP, k = i % NUP;
-                    wv[e] = (j < nu && k < nin) ? Wl[(size_t)(u0 + j) * K + kin0 + k] : __float2bfloat16_rn(0.0f);
-                }
-                const float bv = (tid < NUP && tid < nu) ? m.bias[l][u0 + tid] : 0.0f;
-                // stored source-major, [l][source k][target j]: a new activation updates all its targets
+                    for (int dl = 0; dl < LB; ++dl) {
+                        const int l = min(l0 + dl, L);
+                        const int nu = sh.nu[l], nin = sh.nin[l], u0 = sh.u0[l], kin0 = sh.kin0[l];
+                        const __nv_bfloat16 *Wl = (const __nv_bfloat16 *)m.W[l];
+                        const int K = m.n[l];
 #pragma unroll
-                for (int e = 0; e < NUP * NUP / 128; ++e) {
-                    const int i = tid + e * 128, j = i / NUP, k = i % NUP;
-                    Wg[(l * NUP + k) * NUP + j] = __bfloat162float(wv[e]);
+                        for (int e = 0; e < NUP * NUP / 128; ++e) {
+                            const int i = tid + e * 128, j = i / NUP, k = i % NUP;
+                            wv[dl][e] = (j < nu && k < nin) ? Wl[(size_t)(u0 + j) * K + kin0 + k] : __float2bfloat16_rn(0.0f);
+                        }
+                        bv[dl] = (tid < NUP && tid < nu) ? m.bias[l][u0 + tid] : 0.0f;
+                    }
+                    // weights stored source-major, [l][source k][target j]: a new activation updates all its targets
+#pragma unroll
+                    for (int dl = 0; dl < LB; ++dl) {
+                        const int l = min(l0 + dl, L);           // past the last layer: the last layer again
+#pragma unroll
+                        for (int e = 0; e < NUP * NUP / 128; ++e) {
+                            const int i = tid + e * 128, j = i / NUP, k = i % NUP;
+                            Wg[(l * NUP + k) * NUP + j] = __bfloat162float(wv[dl][e]);
+                        }
+                        if (tid < NUP) sh.bias_s[l][tid] = bv[dl];
+                    }
                 }
-                if (tid < NUP) sh.bias_s[l][tid] = bv;
             }
             {
                 float nv[GMAX];
+                uint8_t xo[GMAX];
                 const float *np = r.noise + (size_t)(valid ? smp : 0) * m.T + t0;
 #pragma unroll
                 for (int i = 0; i < GMAX; ++i) nv[i] = (valid && i < ng) ? __ldg(np + i) : 0.0f;
-#pragma unroll
-                for (int i = 0; i < GMAX; ++i) Nz[i * BM + row] = nv[i];
-            }
-            {
                 // the symbols the group's positions hold now (for the change flags), 255 where there is none
-                uint8_t xo[GMAX];
                 const uint8_t *xp = r.x + (size_t)(valid ? smp : 0) * m.T + t0;
 #pragma unroll
                 for (int i = 0; i < GMAX; ++i) xo[i] = (valid && i < ng) ? xp[i] : (uint8_t)255;
+#pragma unroll
+                for (int i = 0; i < GMAX; ++i) Nz[i * BM + row] = nv[i];
 #pragma unroll
                 for (int i = 0; i < GMAX; ++i) X[i * BM + row] = (float)xo[i];
             }
@@ -458,7 +475,7 @@ struct SweepEngine {
                     for (int c = 0; c * NB < bs.nb && bs.kbs > 0; ++c) {
                         if (!mbar_wait(&sh.bfull[bbuf], (bb_par >> bbuf) & 1u, r.ctl)) { dead = true; break; }
                         tc_fence_after();
-#pragma unroll
+#pragma unroll 1
                         for (int h = 0; h < NB; h += 32) {
                             float v[32];
                             tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(BASE_COL + bbuf * NB + h), v);
@@ -525,7 +542,7 @@ struct SweepEngine {
                 const float enc = sh.lut_s[xn];
                 X[i * BM + row] = enc;
                 if (t + 1 > hi) continue;
-                scatter(0, i, enc, row);
+                scatter(0, i, enc, row, L > 0 ? sh.cs[1][i] - sh.u0[0] : i + 1);
                 // the hidden units that position t makes computable: degree t + 1
                 for (int l = 0; l < L; ++l) {
                     const int j0 = sh.cs[l + 1][i] - sh.u0[l], j1 = sh.cs[l + 1][i + 1] - sh.u0[l];
@@ -533,7 +550,7 @@ struct SweepEngine {
                         const uint32_t pv = vat(l, j, row);
                         const float val = __bfloat162float(__float2bfloat16_rn(tc_act_fn(m.act, lds_f(pv))));
                         sts_f(pv, val);
-                        scatter(l + 1, j, val, row);
+                        scatter(l + 1, j, val, row, l + 1 < L ? sh.cs[l + 2][i] - sh.u0[l + 1] : i + 1);
                     }
                 }
             }
@@ -724,7 +741,7 @@ int js_sweep_prepare(js_model *mo)
     if (sms < 1) return 0;
     s.slots = sms;
     auto fail = [&]() { cudaGetLastError(); return JS_ERR_CUDA; };
-    std::vector<CUtensorMap> mapsF(L + 1), mapsW(3 * (L + 1));       // weights: boxes of 16, of 32 and of 64 rows
+    std::vector<CUtensorMap> mapsF(L + 1), mapsW(3 * (L + 1));       // weights: boxes of 16, of 32 and of NB rows
     for (int l = 0; l <= L; ++l) {
         if (l >= 1) {
             void *p = nullptr;
@@ -751,7 +768,7 @@ int js_sweep_prepare(js_model *mo)
         for (int big = 0; big < 3; ++big) {
             const cuuint64_t dims[2] = {(cuuint64_t)v.n[l], (cuuint64_t)v.n[l + 1]};
             const cuuint64_t strides[1] = {(cuuint64_t)v.n[l] * 2};
-            const cuuint32_t box[2] = {(cuuint32_t)BK, 16u << big};
+            const cuuint32_t box[2] = {(cuuint32_t)BK, big == 2 ? (cuuint32_t)NB : 16u << big};
             if (!sweep_encode(&mapsW[big * (L + 1) + l], v.W[l], 2, dims, strides, box)) return 0;
         }
     }
