@@ -82,6 +82,84 @@ __device__ __forceinline__ float lds_f(uint32_t a)
 }
 __device__ __forceinline__ void sts_f(uint32_t a, float v) { asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory"); }
 
+// Position i of the group when every hidden layer gains exactly one unit there (byte l of jn_packed: its index among
+// the group's units of a[l+1]).  The chain  symbol -> unit of a[1] -> ... -> unit of a[L]  is one scalar
+// fused multiply-add and one activation per layer: the unit's running sum and the one weight are
+// loaded beforehand, so no shared-memory round trip sits between two layers.  The additions to the
+// running sums of everything else in the group (32 per layer) come after the chain, the loads of one
+// layer issued before the arithmetic of the layer below: a warp issues in order, and with one warp
+// per scheduler nothing else hides a load.  Every running sum receives exactly the operations, in
+// exactly the order, of the general path (SweepEngine::scatter).  vbase: the thread's row in slot 0 of V.
+template <int L>
+__device__ __forceinline__ void position_one_each(uint32_t wbase, uint32_t vbase, int act, int i, float enc, int row,
+                                               uint32_t jn_packed)
+{
+    const int sw7 = row & 7;
+    int jn[L];
+#pragma unroll
+    for (int l = 0; l < L; ++l) jn[l] = (int)((jn_packed >> (8 * l)) & 255u);
+    float p[L], ws[L], val[L + 1];
+    uint32_t w4[L + 1], pa[L];
+#pragma unroll
+    for (int l = 0; l <= L; ++l) {
+        const int k = l == 0 ? i : jn[l - 1];                      // this position's source in a[l]
+        w4[l] = wbase + 4u * (uint32_t)((l * NUP + k) * NUP);
+    }
+#pragma unroll
+    for (int l = 0; l < L; ++l) {
+        pa[l] = vbase + 4u * (uint32_t)(l * BM * NUP + ((((jn[l] >> 2) ^ sw7) << 2) | (jn[l] & 3)));
+        p[l] = lds_f(pa[l]);
+        ws[l] = lds_f(w4[l] + 4u * (uint32_t)jn[l]);
+    }
+    val[0] = enc;
+#pragma unroll
+    for (int l = 0; l < L; ++l)
+        val[l + 1] = __bfloat162float(__float2bfloat16_rn(tc_act_fn(act, fmaf(ws[l], val[l], p[l]))));
+    // half a layer (four 16-byte chunks, 16 targets) at a time, two register buffers in turn
+    constexpr int HC = NUP / 8;
+    float4 w[2][HC], x[2][HC];
+    // a half whose 16 targets all lie below the first unit that may read the source is left out (the
+    // same for every thread: the targets' masked weights are zero)
+    bool live[2 * (L + 1)];
+#pragma unroll
+    for (int l = 0; l <= L; ++l) {
+        const int jmin = l < L ? jn[l] : i + 1;
+        live[2 * l] = jmin < 4 * HC;
+        live[2 * l + 1] = true;
+    }
+#pragma unroll
+    for (int h = 0; h <= 2 * (L + 1); ++h) {
+        if (h < 2 * (L + 1) && live[h]) {
+            // loads of half-step h, issued before the arithmetic of half-step h - 1
+            const int l = h >> 1, cb = (h & 1) * HC;
+            const uint32_t v4 = vbase + 4u * (uint32_t)(l * BM * NUP);
+#pragma unroll
+            for (int c = 0; c < HC; ++c)
+                w[h & 1][c] = lds_f4(w4[l] + 16u * (uint32_t)(cb + c));
+#pragma unroll
+            for (int c = 0; c < HC; ++c)
+                x[h & 1][c] = lds_f4(v4 + 16u * (uint32_t)((cb + c) ^ sw7));
+        }
+        if (h >= 1 && live[h - 1]) {
+            const int g = h - 1, l = g >> 1, cb = (g & 1) * HC;
+            const uint32_t v4 = vbase + 4u * (uint32_t)(l * BM * NUP);
+            const float s = val[l];
+#pragma unroll
+            for (int c = 0; c < HC; ++c) {
+                float4 xv = x[g & 1][c];
+                const float4 wv = w[g & 1][c];
+                xv.x = fmaf(wv.x, s, xv.x);
+                xv.y = fmaf(wv.y, s, xv.y);
+                xv.z = fmaf(wv.z, s, xv.z);
+                xv.w = fmaf(wv.w, s, xv.w);
+                sts_f4(v4 + 16u * (uint32_t)((cb + c) ^ sw7), xv);
+            }
+        }
+        // the unit's activation replaces its running sum (after both halves of its layer are stored)
+        if (h >= 1 && ((h - 1) & 1) == 1 && (h - 1) / 2 < L) sts_f(pa[(h - 1) / 2 < L ? (h - 1) / 2 : 0], val[(h - 1) / 2 + 1]);
+    }
+}
+
 struct SweepEngine {
     const MadeDev &m;
     const SweepDev &sw;
@@ -122,7 +200,8 @@ struct SweepEngine {
 
     // optional device timeline (JS_OPT_TRACE, js_get_trace) of the first CTA: one row of stamps per group;
     // slots: 0 operands may be loaded, 1 last MMA issued, 2 group tables ready, 3 prefix sums complete,
-    // 4 prefix sums read, 5 positions done, 6 activations stored
+    // 4 prefix sums read, 5 positions done, 6 activations stored, 7 group geometry ready, 8 the group's
+    // weights staged
     int group_no = 0;
     __device__ void trace(int slot) const
     {
@@ -188,7 +267,7 @@ struct SweepEngine {
         for (int t0 = a; t0 < b && !dead; t0 += sw.G) {
             const int t1 = min(t0 + sw.G, b), hi = min(t1, b - 1);
             // the previous group's activations (or the job's start values) are in F
-            if (!mbar_wait(&sh.gdone, gd_par, r.ctl)) { dead = true; break; }
+            if (!mbar_wait_idle(&sh.gdone, gd_par, r.ctl)) { dead = true; break; }
             gd_par ^= 1u;
             fence_proxy_async();
             trace(0);
@@ -241,7 +320,7 @@ struct SweepEngine {
         for (int t0 = a; t0 < b && !dead; t0 += sw.G) {
             const int t1 = min(t0 + sw.G, b), hi = min(t1, b - 1);
             // the epilogue has read the previous group's accumulators
-            if (!mbar_wait(&sh.tempty, te_par ^ 1u, r.ctl)) { dead = true; break; }
+            if (!mbar_wait_idle(&sh.tempty, te_par ^ 1u, r.ctl)) { dead = true; break; }
             te_par ^= 1u;
             tc_fence_after();
             bool any = false;
@@ -390,6 +469,8 @@ struct SweepEngine {
         if (lane == 0) mbar_arrive(&sh.gdone);
     }
 
+    // LT: the number of hidden layers if the one-unit-per-layer path is compiled for it (1 .. 4), else 0
+    template <int LT>
     __device__ void epilogue(int rt, int slot, int a, int b, bool &row_changed)
     {
         const int q = warp & 3, row = q * 32 + lane, tid = threadIdx.x - 64;
@@ -415,6 +496,7 @@ struct SweepEngine {
                 if (l >= 1) sh.cs[l][k] = cnt(l, min(t0 + k, m.T));
             }
             ep_sync();
+            if (tid == 0) trace(7);
             {
                 // Every global load of the thread first, the stores to shared memory after them: the compiler
                 // may not move a load across a store it cannot tell apart, and one round trip per layer and
@@ -449,6 +531,7 @@ struct SweepEngine {
                     }
                 }
             }
+            if (tid == 0) trace(8);
             {
                 float nv[GMAX];
                 uint8_t xo[GMAX];
@@ -490,6 +573,26 @@ struct SweepEngine {
                     }
                 }
                 if (dead) break;
+            }
+            // ---- the next group's tables (weights between its units, noise, symbols) are touched once per
+            // sweep and would come from DRAM, two dependent round trips of 2.5 us each: ask for them now
+            if (t1 < b) {
+                const int t2 = min(t1 + sw.G, b), hi2 = min(t2, b - 1);
+                for (int i = tid; i < (L + 1) * NUP; i += 128) {
+                    const int l = i / NUP, j = i % NUP;
+                    const Geo g = geo(l, t1, t2, hi2);
+                    if (j < g.nu && g.nin > 0) {
+                        const __nv_bfloat16 *pw = (const __nv_bfloat16 *)m.W[l] + (size_t)(g.u0 + j) * m.n[l] + g.kin0;
+                        prefetch_l2(pw);
+                        prefetch_l2(pw + g.nin - 1);
+                    }
+                }
+                if (valid) {
+                    const float *np = r.noise + (size_t)smp * m.T + t1;
+                    prefetch_l2(np);
+                    prefetch_l2(np + (t2 - t1) - 1);
+                    prefetch_l2(r.x + (size_t)smp * m.T + t1);
+                }
             }
             // ---- prefix sums out of tensor memory
             if (!mbar_wait(&sh.tfull, tf_par, r.ctl)) { dead = true; break; }
@@ -533,15 +636,36 @@ struct SweepEngine {
             // are independent of each other, and each target receives its sources in index order.
             for (int i = 0; i < ng; ++i) {
                 const int t = t0 + i;
+                // the units this position completes, per hidden layer (looked up before the sampling,
+                // which hides the loads)
+                int jn[LT > 0 ? LT : 1];
+                bool one_each = true;
+#pragma unroll
+                for (int l = 0; l < (LT > 0 ? LT : 1); ++l) {
+                    if (LT == 0) break;
+                    const int ca = sh.cs[l + 1][i], cb = sh.cs[l + 1][i + 1];
+                    jn[l] = ca - sh.u0[l];
+                    one_each = one_each && cb - ca == 1;
+                }
                 const float z = lds_f(vat(L, i, row));
-                const int xn = js_sample_binary(r.nk, z, Nz[i * BM + row]);
-                if (valid && (int)X[i * BM + row] != xn) {
+                const uint32_t xa = smem_u32(X) + 4u * (uint32_t)(i * BM + row);
+                const int xn = js_sample_binary(r.nk, z, lds_f(smem_u32(Nz) + 4u * (uint32_t)(i * BM + row)));
+                if (valid && (int)lds_f(xa) != xn) {
                     r.x[(size_t)smp * m.T + t] = (uint8_t)xn;
                     row_changed = true;
                 }
                 const float enc = sh.lut_s[xn];
-                X[i * BM + row] = enc;
+                sts_f(xa, enc);
                 if (t + 1 > hi) continue;
+                if constexpr (LT > 0) {
+                    if (one_each) {
+                        uint32_t pk = 0;                   // indices below 32, one byte each
+#pragma unroll
+                        for (int l = 0; l < LT; ++l) pk |= (uint32_t)jn[l] << (8 * l);
+                        position_one_each<LT>(smem_u32(Wg), smem_u32(V) + 4u * (uint32_t)(row * NUP), m.act, i, enc, row, pk);
+                        continue;
+                    }
+                }
                 scatter(0, i, enc, row, L > 0 ? sh.cs[1][i] - sh.u0[0] : i + 1);
                 // the hidden units that position t makes computable: degree t + 1
                 for (int l = 0; l < L; ++l) {
@@ -573,6 +697,9 @@ struct SweepEngine {
     }
 };
 
+// LT = the model's number of hidden layers where the one-unit-per-layer path of the position loop is
+// compiled for it (1 .. 4), else 0.
+template <int LT>
 __global__ void __launch_bounds__(NTH, 1)
 made_sweep_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ SweepDev sw, const __grid_constant__ RunArgs r)
 {
@@ -617,7 +744,7 @@ made_sweep_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ Swe
             if (e.lane == 0) e.mma_issuer(a, b);
         } else {
             bool row_changed = false;
-            e.epilogue(rt, blockIdx.x, a, b, row_changed);
+            e.template epilogue<LT>(rt, blockIdx.x, a, b, row_changed);
             const int smp = rt * BM + (warp & 3) * 32 + e.lane;
             if (row_changed && smp < r.batch) r.smp_changed[smp] = 1;
         }
@@ -691,6 +818,18 @@ static bool sweep_encode(CUtensorMap *out, const void *base, int rank, const cuu
     return fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+typedef void (*SweepKernelFn)(const MadeDev, const SweepDev, const RunArgs);
+static SweepKernelFn sweep_kernel_of(int L)
+{
+    switch (L) {
+    case 1: return made_sweep_kernel<1>;
+    case 2: return made_sweep_kernel<2>;
+    case 3: return made_sweep_kernel<3>;
+    case 4: return made_sweep_kernel<4>;
+    default: return made_sweep_kernel<0>;
+    }
 }
 
 // Builds what the sweeps need beside the tensor-core view of the model: prefix counts per degree,
@@ -804,7 +943,7 @@ int js_sweep_prepare(js_model *mo)
         if (cudaHostAlloc((void **)&mo->h_any, sizeof(int), cudaHostAllocMapped) != cudaSuccess) return fail();
         if (cudaHostGetDevicePointer((void **)&mo->d_any, mo->h_any, 0) != cudaSuccess) return fail();
     }
-    if (cudaFuncSetAttribute(made_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_MAX) != cudaSuccess) {
+    if (cudaFuncSetAttribute(sweep_kernel_of(L), cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_DYN_MAX) != cudaSuccess) {
         cudaGetLastError();
         return 0;
     }
@@ -820,7 +959,7 @@ int js_launch_made_sweep(const js_model *mo, const RunArgs &r, cudaStream_t stre
     const int njobs = MT * (nblk - r.blk_lo);
     if (njobs < 1) return (int)cudaErrorInvalidValue;
     const int grid = std::min(njobs, s.slots);
-    made_sweep_kernel<<<grid, NTH, s.smem_bytes, stream>>>(mo->made, s, r);
+    sweep_kernel_of(mo->made.L)<<<grid, NTH, s.smem_bytes, stream>>>(mo->made, s, r);
     const cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? 0 : (int)e;
 }

@@ -60,6 +60,25 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, JsCtl 
     return false;
 }
 
+// The same for waits that are expected to last tens of microseconds while other warps of the CTA work out
+// of shared memory: polls 0.1 us apart, so that the waiting lane leaves the issue slots and the
+// shared-memory pipe to them.
+__device__ __forceinline__ bool mbar_wait_idle(uint64_t *bar, uint32_t parity, JsCtl *ctl)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_ns();
+    for (unsigned i = 1;; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        __nanosleep(100);
+        if ((i & 63u) == 0u) {
+            if (ld_volatile_i32(&ctl->abort) != 0) break;
+            if (global_ns() - t0 > MBAR_WAIT_NS) break;
+        }
+    }
+    atomicExch(&ctl->abort, 1);
+    return false;
+}
+
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1)
 {
     asm volatile(
