@@ -206,3 +206,59 @@ def conv_weights(cfg: ConvConfig, salt: int = 0):
 def conv_lut(cfg: ConvConfig) -> np.ndarray:
     n = cfg.C
     return (np.arange(n, dtype=np.float64) / ((n - 1) / 2.0) - 1.0).astype(np.float32)
+
+
+# ---------------------------------------------------------------- recurrent-network workload
+@dataclass(frozen=True)
+class RnnConfig:
+    """Shape of the recurrent-network workload (back-propagation through time, Section 5.1)."""
+    name: str
+    index: int                 # fixes the seeds
+    T: int = 100               # sequence length: a 10x10 image, one pixel per step
+    H: int = 128               # hidden units
+    d_in: int = 1
+    d_out: int = 1
+    batch: int = 1             # independent sequences
+    w_std: float = 0.1         # weights ~ N(0, w_std^2), biases zero
+    kind: str = "rnn"
+
+
+# The paper trains on MNIST digits resized to 10x10 and fed pixel by pixel; seeded images of a few
+# soft strokes on a 10x10 grid stand in for them (same length, same value range, same smoothness).
+RNN_CONFIGS: Dict[str, RnnConfig] = {
+    "rnn_small": RnnConfig("rnn_small", 10, T=12, H=16, batch=3),
+    "rnn_100": RnnConfig("rnn_100", 11, T=100, H=128, batch=1),
+    "rnn_100_batch": RnnConfig("rnn_100_batch", 12, T=100, H=128, batch=592),
+}
+
+
+def rnn_weights(cfg: RnnConfig):
+    """(W_h [H,H], W_x [H,d_in], b [H], W_o [d_out,H], b_o [d_out]) as float32."""
+    rng = _rng(cfg, 0)
+    var = cfg.w_std * cfg.w_std
+    Wh = _normal(rng, (cfg.H, cfg.H), var)
+    Wx = _normal(rng, (cfg.H, cfg.d_in), var)
+    Wo = _normal(rng, (cfg.d_out, cfg.H), var)
+    return Wh, Wx, np.zeros(cfg.H, np.float32), Wo, np.zeros(cfg.d_out, np.float32)
+
+
+def rnn_sequences(cfg: RnnConfig):
+    """Inputs x [batch, T, d_in] in [0, 1] and targets r [batch, T, d_out] (the next input, zero after
+    the last step), float32."""
+    rng = _rng(cfg, 2)
+    side = int(np.ceil(np.sqrt(cfg.T)))
+    yy, xx = np.mgrid[0:side, 0:side].astype(np.float64)
+    x = np.zeros((cfg.batch, cfg.T, cfg.d_in), np.float32)
+    for b in range(cfg.batch):
+        for c in range(cfg.d_in):
+            img = np.zeros((side, side))
+            for _ in range(3):                       # three soft strokes
+                cy, cx = rng.uniform(1.0, side - 2.0, size=2)
+                sy, sx = rng.uniform(0.6, 2.0, size=2)
+                img += np.exp(-0.5 * (((yy - cy) / sy) ** 2 + ((xx - cx) / sx) ** 2))
+            img = np.clip(img, 0.0, 1.0)
+            x[b, :, c] = img.reshape(-1)[:cfg.T].astype(np.float32)
+    r = np.zeros((cfg.batch, cfg.T, cfg.d_out), np.float32)
+    n = min(cfg.d_in, cfg.d_out)
+    r[:, :-1, :n] = x[:, 1:, :n]
+    return x, r
