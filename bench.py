@@ -419,6 +419,74 @@ def cpu_leg(cfg, inputs, mode_name, block, n, gpu_samples, gpu_iters):
             "samples_differing_from_gpu": differing}
 
 
+def measure_rnn(local: int, with_oracle: bool):
+    """The recurrent-network workload (Section 5.1): gradients of a batch of sequences, the backward pass by
+    back-substitution and by Jacobi_n.  Times are CUDA-event means over 20 calls after 3 warm-up calls; the
+    inputs stay resident and L2 is flushed between calls."""
+    import torch
+    import paper_2002_03629_b200.rnn as rnn
+    out = {}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for name in ("rnn_100", "rnn_100_batch"):
+        cfg = si.RNN_CONFIGS[name]
+        params = [torch.from_numpy(a).cuda() for a in si.rnn_weights(cfg)]
+        x, r = (torch.from_numpy(a).cuda() for a in si.rnn_sequences(cfg))
+        h, d, l, loss = rnn.rnn_forward(*params, x, r)
+        s = torch.empty_like(l)
+
+        def timed(fn, reps=20):
+            for _ in range(3):
+                fn()
+            tot = 0.0
+            for _ in range(reps):
+                flush.fill_(1)
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn()
+                b.record()
+                b.synchronize()
+                tot += a.elapsed_time(b)
+            return tot / reps
+
+        rec = {"batch": cfg.batch, "T": cfg.T, "H": cfg.H, "dtype": "f32",
+               "forward_ms": timed(lambda: rnn.rnn_forward(*params, x, r)),
+               "backward_sequential_ms": timed(lambda: rnn.rnn_bptt_sequential(params[0], l, d, out=s)),
+               "param_grads_ms": timed(lambda: rnn.rnn_param_grads(s, d, h, x))}
+        exact = rnn.rnn_bptt_sequential(params[0], l, d)
+        for n in (5, 10, 20, cfg.T):
+            ms = timed(lambda: rnn.rnn_bptt_jacobi(params[0], l, d, n, out=s))
+            sn = rnn.rnn_bptt_jacobi(params[0], l, d, n)
+            err = ((sn - exact).norm() / exact.norm()).item()
+            flops = 2.0 * cfg.batch * n * cfg.T * cfg.H * cfg.H
+            rec[f"backward_jacobi_{n}"] = {"ms": ms, "rel_l2_error_vs_exact": err, "tflops": flops / ms / 1e9}
+        # fp32 fused multiply-add peak: SMs x 128 lanes x 2 flop x clock
+        prop = torch.cuda.get_device_properties(local)
+        peak = prop.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
+        j = rec[f"backward_jacobi_{cfg.T}"]
+        rec["roofline"] = {"bound": "alu", "kernel": "rnn_bptt_jacobi_kernel", "achieved": j["tflops"], "peak": peak,
+                           "unit": "TFLOP/s", "frac": j["tflops"] / peak,
+                           "peak_source": "SMs x 128 fp32 lanes x 2 x 1965 MHz (nominal; derived, not measured)"}
+        rec["sequences_per_s_exact_gradient"] = cfg.batch / ((rec["forward_ms"] + rec["backward_sequential_ms"] +
+                                                              rec["param_grads_ms"]) / 1e3)
+        if with_oracle:
+            from oracle import rnn_oracle as ro
+            Wn = [p_.cpu().numpy() for p_ in params]
+            xs, rs = x.cpu().numpy(), r.cpu().numpy()
+            k = min(cfg.batch, 8)
+            t0 = time.perf_counter()
+            worst = 0.0
+            for i in range(k):
+                f = ro.forward(*Wn, xs[i], rs[i])
+                se = ro.backprop_exact(Wn[0], f["l"], f["d"])
+                ro.param_grads(se, f["d"], f["h"], xs[i])
+                worst = max(worst, float(np.abs(exact[i].cpu().double().numpy() - se).max() / np.abs(se).max()))
+            dt = time.perf_counter() - t0
+            rec["oracle"] = {"sample": f"{k} sequences, forward + exact backward + parameter gradients, numpy float64, 1 thread",
+                             "sequences_per_s": k / dt, "max_rel_error_of_gpu_exact_states": worst}
+        out[name] = rec
+    return out
+
+
 def oracle_sample_count(cfg, budget_s):
     cores = os.cpu_count() or 1
     per_sample_s = (14.0 if cfg.kind == "conv" else 4.0) * live_macs_per_sample(cfg) / 0.6e9
@@ -495,6 +563,8 @@ def run_ours(args, cfg):
                                                    "samples_differing_from_gpu")}
             wl[name] = r2
             del ex2, in2
+        # the recurrent-network workload (another instance of the same triangular-system view)
+        wl.update(measure_rnn(local, not args.no_cpu_baseline))
         line["workloads"] = wl
     print(json.dumps(line))
     if world > 1:

@@ -10,16 +10,21 @@ LIB = os.path.join(HERE, "libjacobi_sample.so")
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 
 
+def _tree():
+    """Every file under csrc/ (the sampler's kernels at the top, the recurrent-network workload in rnn/)."""
+    return sorted(os.path.join(d, f) for d, _, fs in os.walk(CSRC) for f in fs)
+
+
 def sources():
-    return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".cu"))
+    return [f for f in _tree() if f.endswith(".cu")]
 
 
 def _stale() -> bool:
     if not os.path.exists(LIB):
         return True
     t = os.path.getmtime(LIB)
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)]
-    deps.append(os.path.join(os.path.dirname(HERE), "include", "jacobi_sample.h"))
+    inc = os.path.join(os.path.dirname(HERE), "include")
+    deps = _tree() + [os.path.join(inc, f) for f in os.listdir(inc)]
     return any(os.path.getmtime(d) > t for d in deps)
 
 

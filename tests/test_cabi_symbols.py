@@ -9,7 +9,8 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
 def declared_symbols():
-    text = open(os.path.join(ROOT, "include", "jacobi_sample.h")).read()
+    inc = os.path.join(ROOT, "include")
+    text = "\n".join(open(os.path.join(inc, f)).read() for f in sorted(os.listdir(inc)) if f.endswith(".h"))
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     names = re.findall(r"^\s*(?:const\s+)?[A-Za-z_][\w\s\*]*?\b(\w+)\s*\([^;{]*\)\s*;", text, flags=re.M)
     return sorted(set(names))
@@ -20,7 +21,8 @@ def test_header_declares_the_entry_points():
     for must in ("jacobi_sample", "sequential_sample", "js_made_create", "js_conv_create", "js_model_destroy",
                  "js_forward_logits", "js_set_option", "js_get_stats", "js_strerror", "js_last_cuda_error",
                  "jacobi_sample_host", "jacobi_sample_real", "sequential_sample_real", "js_forward_logits_real",
-                 "jacobi_sample_noalloc", "js_get_trace"):
+                 "jacobi_sample_noalloc", "js_get_trace", "rnn_forward", "rnn_bptt_sequential", "rnn_bptt_jacobi",
+                 "rnn_param_grads", "rnn_last_error"):
         assert must in names, names
 
 
