@@ -253,7 +253,7 @@ def rnn_sequences(cfg: RnnConfig):
         for c in range(cfg.d_in):
             img = np.zeros((side, side))
             for _ in range(3):                       # three soft strokes
-                cy, cx = rng.uniform(1.0, side - 2.0, size=2)
+                cy, cx = rng.uniform(min(1.0, side - 1.0), max(side - 2.0, min(1.0, side - 1.0)), size=2)
                 sy, sx = rng.uniform(0.6, 2.0, size=2)
                 img += np.exp(-0.5 * (((yy - cy) / sy) ** 2 + ((xx - cx) / sx) ** 2))
             img = np.clip(img, 0.0, 1.0)
