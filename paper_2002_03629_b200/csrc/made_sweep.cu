@@ -44,6 +44,7 @@ constexpr int GPB = 8;                       // groups per base: a base GEMM ser
 constexpr int W_BYTES = NB * BK * 2;
 constexpr int STAGE_BYTES = A_BYTES + W_BYTES;          // 32 KB, a multiple of 1 KB
 constexpr int BASE_COL = 256;                // tensor-memory columns of the two base accumulators (NB each)
+constexpr int XS = BM + 1;                    // row stride of X and Nz: a lane per position writes without bank conflicts
 constexpr int MAX_STAGES = 10;
 constexpr int SMEM_DYN_MAX = 227 * 1024 - 4 * 1024;
 
@@ -100,16 +101,18 @@ __device__ __forceinline__ void position_one_each(uint32_t wbase, uint32_t vbase
     for (int l = 0; l < L; ++l) jn[l] = (int)((jn_packed >> (8 * l)) & 255u);
     float p[L], ws[L], val[L + 1];
     uint32_t w4[L + 1], pa[L];
+    int kw7[L + 1];                                                 // the weight rows' chunk permutation
 #pragma unroll
     for (int l = 0; l <= L; ++l) {
         const int k = l == 0 ? i : jn[l - 1];                      // this position's source in a[l]
         w4[l] = wbase + 4u * (uint32_t)((l * NUP + k) * NUP);
+        kw7[l] = k & 7;
     }
 #pragma unroll
     for (int l = 0; l < L; ++l) {
         pa[l] = vbase + 4u * (uint32_t)(l * BM * NUP + ((((jn[l] >> 2) ^ sw7) << 2) | (jn[l] & 3)));
         p[l] = lds_f(pa[l]);
-        ws[l] = lds_f(w4[l] + 4u * (uint32_t)jn[l]);
+        ws[l] = lds_f(w4[l] + 4u * (uint32_t)((((jn[l] >> 2) ^ kw7[l]) << 2) | (jn[l] & 3)));
     }
     val[0] = enc;
 #pragma unroll
@@ -135,7 +138,7 @@ __device__ __forceinline__ void position_one_each(uint32_t wbase, uint32_t vbase
             const uint32_t v4 = vbase + 4u * (uint32_t)(l * BM * NUP);
 #pragma unroll
             for (int c = 0; c < HC; ++c)
-                w[h & 1][c] = lds_f4(w4[l] + 16u * (uint32_t)(cb + c));
+                w[h & 1][c] = lds_f4(w4[l] + 16u * (uint32_t)((cb + c) ^ kw7[l]));
 #pragma unroll
             for (int c = 0; c < HC; ++c)
                 x[h & 1][c] = lds_f4(v4 + 16u * (uint32_t)((cb + c) ^ sw7));
@@ -168,9 +171,9 @@ struct SweepEngine {
     uint8_t *ring;
     float *V;            // [L+1][128 rows][NUP]: running sums, then activations, of the group's units; a row's
                          // eight 16-byte chunks are permuted by the row number (conflict-free 16-byte accesses)
-    float *X;            // [NUP][128]: encodings of the group's positions
+    float *X;            // [NUP][XS]: encodings of the group's positions
     float *Wg;           // [L+1][NUP][NUP]: weights between the group's units
-    float *Nz;           // [GMAX][128]: the group's noise
+    float *Nz;           // [GMAX][XS]: the group's noise
     int warp, lane;
     int stage = 0;
     uint32_t spar = 0;
@@ -192,7 +195,7 @@ struct SweepEngine {
         V = reinterpret_cast<float *>(ring);
         uint8_t *p = ring + (size_t)sw.ring_bytes;
         X = reinterpret_cast<float *>(p);
-        p += (size_t)NUP * BM * 4;
+        p += (size_t)NUP * XS * 4;
         Wg = reinterpret_cast<float *>(p);
         p += (size_t)(m.L + 1) * NUP * NUP * 4;
         Nz = reinterpret_cast<float *>(p);
@@ -382,6 +385,10 @@ struct SweepEngine {
         }
     }
 
+    // row k (a source among the group's units of a[l]) of the table of weights inside the group: 32 targets
+    // as eight 16-byte chunks, chunk c stored at position c ^ (k & 7)
+    __device__ uint32_t wrow(int l, int k) const { return smem_u32(Wg) + 4u * (uint32_t)((l * NUP + k) * NUP); }
+
     __device__ void ep_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
     // unit j of the group in layer slot l, sample row `row`: its shared-memory address
@@ -399,13 +406,13 @@ struct SweepEngine {
         const int c0 = jmin >> 2;
         // the row's 32 running sums as eight 16-byte accesses, all loads before all stores: one warp per
         // scheduler cannot hide the latency of a load that waits behind a store it might alias
-        const uint32_t w4 = smem_u32(Wg) + 4u * (uint32_t)((l * NUP + k) * NUP);
+        const uint32_t w4 = wrow(l, k);
         const uint32_t v4 = smem_u32(V) + 4u * (uint32_t)((l * BM + row) * NUP);
-        const int sw7 = row & 7;
+        const int sw7 = row & 7, kw7 = k & 7;
         float4 w[NUP / 4], x[NUP / 4];
 #pragma unroll
         for (int c = 0; c < NUP / 4; ++c)
-            if (c >= c0) w[c] = lds_f4(w4 + 16u * c);
+            if (c >= c0) w[c] = lds_f4(w4 + 16u * (uint32_t)(c ^ kw7));
 #pragma unroll
         for (int c = 0; c < NUP / 4; ++c)
             if (c >= c0) x[c] = lds_f4(v4 + 16u * (uint32_t)(c ^ sw7));
@@ -424,7 +431,7 @@ struct SweepEngine {
 
     // n consecutive values (unit j = 0..n-1 of layer slot l, or the group's encodings when l < 0) of this
     // thread's row as bf16 to dst[0..n): single elements up to a 16-byte boundary, then eight at a time
-    __device__ float run_val(int l, int j, int row) const { return l < 0 ? X[j * BM + row] : lds_f(vat(l, j, row)); }
+    __device__ float run_val(int l, int j, int row) const { return l < 0 ? X[j * XS + row] : lds_f(vat(l, j, row)); }
     __device__ void store_run(__nv_bfloat16 *dst, int l, int row, int n)
     {
         int j = 0;
@@ -501,9 +508,12 @@ struct SweepEngine {
                 // Every global load of the thread first, the stores to shared memory after them: the compiler
                 // may not move a load across a store it cannot tell apart, and one round trip per layer and
                 // per table would cost more than the group's GEMMs.
+                // thread = (source k = lane, chunk of four targets): four loads (each coalesced over the
+                // warp's sources), one 16-byte store to row k of the source-major table, chunks permuted by
+                // the row number like the running sums (a new activation updates all its targets)
                 constexpr int LB = 3;            // layers per round trip
                 for (int l0 = 0; l0 <= L; l0 += LB) {
-                    __nv_bfloat16 wv[LB][NUP * NUP / 128];
+                    __nv_bfloat16 wv[LB][2][4];
                     float bv[LB];
 #pragma unroll
                     for (int dl = 0; dl < LB; ++dl) {
@@ -512,40 +522,49 @@ struct SweepEngine {
                         const __nv_bfloat16 *Wl = (const __nv_bfloat16 *)m.W[l];
                         const int K = m.n[l];
 #pragma unroll
-                        for (int e = 0; e < NUP * NUP / 128; ++e) {
-                            const int i = tid + e * 128, j = i / NUP, k = i % NUP;
-                            wv[dl][e] = (j < nu && k < nin) ? Wl[(size_t)(u0 + j) * K + kin0 + k] : __float2bfloat16_rn(0.0f);
-                        }
+                        for (int e = 0; e < 2; ++e)
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj) {
+                                const int j = 4 * (q + 4 * e) + jj;
+                                wv[dl][e][jj] = (j < nu && lane < nin) ? Wl[(size_t)(u0 + j) * K + kin0 + lane]
+                                                                       : __float2bfloat16_rn(0.0f);
+                            }
                         bv[dl] = (tid < NUP && tid < nu) ? m.bias[l][u0 + tid] : 0.0f;
                     }
-                    // weights stored source-major, [l][source k][target j]: a new activation updates all its targets
 #pragma unroll
                     for (int dl = 0; dl < LB; ++dl) {
                         const int l = min(l0 + dl, L);           // past the last layer: the last layer again
 #pragma unroll
-                        for (int e = 0; e < NUP * NUP / 128; ++e) {
-                            const int i = tid + e * 128, j = i / NUP, k = i % NUP;
-                            Wg[(l * NUP + k) * NUP + j] = __bfloat162float(wv[dl][e]);
-                        }
+                        for (int e = 0; e < 2; ++e)
+                            sts_f4(wrow(l, lane) + 16u * (uint32_t)((q + 4 * e) ^ (lane & 7)),
+                                   make_float4(__bfloat162float(wv[dl][e][0]), __bfloat162float(wv[dl][e][1]),
+                                               __bfloat162float(wv[dl][e][2]), __bfloat162float(wv[dl][e][3])));
                         if (tid < NUP) sh.bias_s[l][tid] = bv[dl];
                     }
                 }
             }
             if (tid == 0) trace(8);
             {
-                float nv[GMAX];
-                uint8_t xo[GMAX];
-                const float *np = r.noise + (size_t)(valid ? smp : 0) * m.T + t0;
+                // noise and the symbols the group's positions hold now (for the change flags; 255 where there
+                // is none): a warp takes its 32 rows in turn, lane = position, so that a load instruction
+                // touches one line instead of 32; eight rows' loads before their stores
+#pragma unroll 1
+                for (int r0 = 0; r0 < 32; r0 += 8) {
+                    float nv[8];
+                    uint8_t xo[8];
 #pragma unroll
-                for (int i = 0; i < GMAX; ++i) nv[i] = (valid && i < ng) ? __ldg(np + i) : 0.0f;
-                // the symbols the group's positions hold now (for the change flags), 255 where there is none
-                const uint8_t *xp = r.x + (size_t)(valid ? smp : 0) * m.T + t0;
+                    for (int rr = 0; rr < 8; ++rr) {
+                        const int s2 = rt * BM + q * 32 + r0 + rr;
+                        const bool in = s2 < r.batch && lane < ng;
+                        nv[rr] = in ? __ldg(r.noise + (size_t)s2 * m.T + t0 + lane) : 0.0f;
+                        xo[rr] = in ? r.x[(size_t)s2 * m.T + t0 + lane] : (uint8_t)255;
+                    }
 #pragma unroll
-                for (int i = 0; i < GMAX; ++i) xo[i] = (valid && i < ng) ? xp[i] : (uint8_t)255;
-#pragma unroll
-                for (int i = 0; i < GMAX; ++i) Nz[i * BM + row] = nv[i];
-#pragma unroll
-                for (int i = 0; i < GMAX; ++i) X[i * BM + row] = (float)xo[i];
+                    for (int rr = 0; rr < 8; ++rr) {
+                        Nz[lane * XS + q * 32 + r0 + rr] = nv[rr];
+                        X[lane * XS + q * 32 + r0 + rr] = (float)xo[rr];
+                    }
+                }
             }
             ep_sync();
             if (tid == 0) trace(2);
@@ -648,8 +667,8 @@ struct SweepEngine {
                     one_each = one_each && cb - ca == 1;
                 }
                 const float z = lds_f(vat(L, i, row));
-                const uint32_t xa = smem_u32(X) + 4u * (uint32_t)(i * BM + row);
-                const int xn = js_sample_binary(r.nk, z, lds_f(smem_u32(Nz) + 4u * (uint32_t)(i * BM + row)));
+                const uint32_t xa = smem_u32(X) + 4u * (uint32_t)(i * XS + row);
+                const int xn = js_sample_binary(r.nk, z, lds_f(smem_u32(Nz) + 4u * (uint32_t)(i * XS + row)));
                 if (valid && (int)lds_f(xa) != xn) {
                     r.x[(size_t)smp * m.T + t] = (uint8_t)xn;
                     row_changed = true;
@@ -681,10 +700,25 @@ struct SweepEngine {
             if (tid == 0) trace(5);
             // ---- the group's activations into F, for the GEMMs of the groups that follow
             if (t1 < b) {
+                // the symbols' encodings by thread = row (their table is position-major); the hidden
+                // units by warp: its 32 rows in turn, lane = unit, so that a store instruction writes one
+                // run of 2-byte values instead of touching 32 lines
                 store_run(sw.F[0] + ((size_t)slot * BM + row) * sw.WF[0] + (t0 - kb_old[0] * BK), -1, row, ng);
-                for (int l = 1; l <= L; ++l)
-                    store_run(sw.F[l] + ((size_t)slot * BM + row) * sw.WF[l] + (sh.kin0[l] - kb_old[l] * BK), l - 1, row,
-                              sh.nin[l]);
+                __syncwarp();
+                for (int l = 1; l <= L; ++l) {
+                    const int n = sh.nin[l];
+                    __nv_bfloat16 *dst = sw.F[l] + ((size_t)slot * BM + q * 32) * sw.WF[l] + (sh.kin0[l] - kb_old[l] * BK) + lane;
+                    if (lane < n) {
+#pragma unroll 1
+                        for (int r0 = 0; r0 < 32; r0 += 8) {
+                            float v[8];
+#pragma unroll
+                            for (int rr = 0; rr < 8; ++rr) v[rr] = lds_f(vat(l - 1, lane, q * 32 + r0 + rr));
+#pragma unroll
+                            for (int rr = 0; rr < 8; ++rr) dst[(size_t)(r0 + rr) * sw.WF[l]] = __float2bfloat16_rn(v[rr]);
+                        }
+                    }
+                }
                 fence_proxy_async();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sh.gdone);
@@ -868,7 +902,7 @@ int js_sweep_prepare(js_model *mo)
     if (G < 1) return 0;
     s.G = G;
     const int v_bytes = (L + 1) * NUP * BM * 4;            // shares the ring's memory
-    const int fixed = NUP * BM * 4 + (L + 1) * NUP * NUP * 4 + GMAX * BM * 4;
+    const int fixed = NUP * XS * 4 + (L + 1) * NUP * NUP * 4 + GMAX * XS * 4;
     s.n_stages = std::min(MAX_STAGES, (SMEM_DYN_MAX - 1024 - fixed) / STAGE_BYTES);
     if (s.n_stages < 2) return 0;
     s.ring_bytes = std::max(s.n_stages * STAGE_BYTES, (v_bytes + 1023) / 1024 * 1024);
