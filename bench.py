@@ -487,6 +487,77 @@ def measure_rnn(local: int, with_oracle: bool):
     return out
 
 
+def measure_real(pkg, local: int, with_oracle: bool):
+    """Continuous states with logistic conditionals (Section 5.3.1, Appendix C.3): Jacobi with the stopping
+    tolerance eps on the largest change, and with eps = 0, beside the strict order on the same kernels
+    (CUDA-core path, fp32).  CUDA-event means over 10 calls after 3 warm-up calls, inputs resident, L2 flushed
+    between calls."""
+    import torch
+    out = {}
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for name, cfg in si.REAL_CONFIGS.items():
+        W, b = si.made_real_weights(cfg)
+        lut = np.zeros(2, np.float32)
+        model = pkg.Model.made(cfg.D, 2, list(cfg.H), cfg.act, cfg.prec, W, b, lut, cfg.batch)
+        noise = si.draw_noise(cfg)
+        d_noise = torch.from_numpy(noise).cuda()
+        x = torch.empty((cfg.batch, cfg.D), dtype=torch.float32, device="cuda")
+        it = torch.empty((cfg.batch,), dtype=torch.int32, device="cuda")
+
+        def timed(fn, reps=10):
+            for _ in range(3):
+                fn()
+            tot = 0.0
+            for _ in range(reps):
+                flush.fill_(1)
+                a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn()
+                e.record()
+                e.synchronize()
+                tot += a.elapsed_time(e)
+            return tot / reps
+
+        rec = {"batch": cfg.batch, "T": cfg.D, "hidden": list(cfg.H), "dtype": "f32", "kernel_path": "cuda-core"}
+        macs = live_macs_per_sample(cfg)
+        for key, eps in (("jacobi_eps", si.REAL_EPS), ("jacobi_exact", 0.0)):
+            ms = timed(lambda: pkg.jacobi_sample_real(model, d_noise, None, pkg.JS_JACOBI, 0, 0, eps, x, it))
+            st = model.stats()
+            it_np = it.cpu().numpy()
+            rec[key] = {"eps": eps, "ms_per_call": ms, "samples_per_s": cfg.batch / ms * 1e3,
+                        "iters_per_sample": {"mean": float(it_np.mean()), "max": int(it_np.max()),
+                                             "forward_passes": int(st.iterations)},
+                        "tflops_live": 2.0 * macs * float(it_np.sum()) / ms / 1e9}
+            if key == "jacobi_eps":
+                x_eps, it_eps = x.cpu().numpy(), it_np
+        seq = torch.empty_like(x)
+        ms_seq = timed(lambda: pkg.sequential_sample_real(model, d_noise, seq), reps=3)
+        rec["sequential_on_gpu"] = {"ms": ms_seq, "us_per_position": ms_seq * 1e3 / cfg.D,
+                                    "largest_distance_to_jacobi_exact": float((seq - x).abs().max().item())}
+        rec["speedup_vs_sequential"] = {"jacobi_eps": ms_seq / rec["jacobi_eps"]["ms_per_call"],
+                                        "jacobi_exact": ms_seq / rec["jacobi_exact"]["ms_per_call"]}
+        prop = torch.cuda.get_device_properties(local)
+        peak = prop.multi_processor_count * 128 * 2 * 1.965e9 / 1e12
+        rec["roofline"] = {"bound": "alu", "kernel": "made_generic_kernel", "achieved": rec["jacobi_eps"]["tflops_live"],
+                           "peak": peak, "unit": "TFLOP/s", "frac": rec["jacobi_eps"]["tflops_live"] / peak,
+                           "peak_source": "SMs x 128 fp32 lanes x 2 x 1965 MHz (nominal; derived, not measured)"}
+        if with_oracle:
+            from oracle import Oracle
+            orc = Oracle.made(cfg.D, 2, list(cfg.H), cfg.act, cfg.prec, W, b, lut)
+            k = min(cfg.batch, 32)
+            t0 = time.perf_counter()
+            ref = [orc.jacobi_real(noise[i], si.REAL_EPS) for i in range(k)]
+            dt = time.perf_counter() - t0
+            rec["oracle"] = {"sample": f"{k} of {cfg.batch} samples, jacobi with eps {si.REAL_EPS}, 1 thread, {dt:.1f} s",
+                             "samples_per_s": k / dt,
+                             "iters_per_sample_mean": float(np.mean([r[1] for r in ref])),
+                             "gpu_iters_mean_on_same_samples": float(it_eps[:k].mean()),
+                             "largest_state_difference": float(max(np.abs(ref[i][0] - x_eps[i]).max() for i in range(k)))}
+        model.close()
+        out[name] = rec
+    return out
+
+
 def oracle_sample_count(cfg, budget_s):
     cores = os.cpu_count() or 1
     per_sample_s = (14.0 if cfg.kind == "conv" else 4.0) * live_macs_per_sample(cfg) / 0.6e9
@@ -565,6 +636,8 @@ def run_ours(args, cfg):
             del ex2, in2
         # the recurrent-network workload (another instance of the same triangular-system view)
         wl.update(measure_rnn(local, not args.no_cpu_baseline))
+        # continuous states with a stopping tolerance
+        wl.update(measure_real(pkg, local, not args.no_cpu_baseline))
         line["workloads"] = wl
     print(json.dumps(line))
     if world > 1:

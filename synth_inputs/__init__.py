@@ -104,6 +104,25 @@ CONFIGS: Dict[str, object] = {
 CONFIGS["made_cat_icdf"] = replace(CONFIGS["made_cat"], name="made_cat_icdf", noise_kind=NOISE_UNIFORM_CAT)
 
 
+# continuous states (logistic conditionals: a location and a log-scale per position, C = 2): config 2's shape
+# with fp32 weights; stopping tolerance of the solvers in REAL_EPS
+REAL_CONFIGS: Dict[str, MadeConfig] = {
+    "made_784_real": MadeConfig("made_784_real", 7, D=784, C=2, H=(1024, 1024), act=ACT_RELU, prec=PREC_F32,
+                                batch=256, noise_kind=NOISE_LOGISTIC, w_var_scale=2.0, b_var=0.05),
+}
+REAL_EPS = 0.01
+
+
+def made_real_weights(cfg: MadeConfig, salt: int = 0):
+    """Weights of a network with continuous states: the rows of the output layer that produce log-scales are
+    damped (a quarter of the weight, bias shifted by -1), so that the conditionals stay narrow enough for the
+    fixed-point iteration to settle in a few dozen steps."""
+    W, b = made_weights(cfg, salt)
+    W[-1][1::2] *= np.float32(0.25)
+    b[-1][1::2] -= np.float32(1.0)
+    return W, b
+
+
 def scaled(cfg, **changes):
     """A smaller workload with the same structure (used by parity tests)."""
     return replace(cfg, **changes)
