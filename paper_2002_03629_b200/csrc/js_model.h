@@ -15,6 +15,7 @@ struct TcLayer {
     int bn;
     int nt;
     int stage_bytes, n_stages;   // this layer's cut of the operand ring
+    int npad;                    // units padded to whole tiles: rows per K block of the tile-major weight copy
     // split-K: the K blocks of tile nt are cut into chunks of `ch` blocks, each chunk a work unit
     // of its own; the last chunk owns the tile and adds the others' fp32 partial sums in order
     int ch;

@@ -338,7 +338,7 @@ struct TcEngine {
                 if (!mbar_wait(&sh.empty[stage], stage_parity() ^ 1u, r.ctl)) { dead = true; break; }
                 mbar_expect_tx(&sh.full[stage], bytes);
                 tma_load_2d(smem_u32(stage_a(stage)), ma, &sh.full[stage], kb * BK, u.mt * BM);
-                tma_load_2d(smem_u32(stage_b(stage)), mw, &sh.full[stage], kb * BK, u.nt * ly.bn);
+                tma_load_2d(smem_u32(stage_b(stage)), mw, &sh.full[stage], 0, kb * ly.npad + u.nt * ly.bn);
                 advance_stage();
             }
         }
@@ -354,7 +354,7 @@ struct TcEngine {
             Unit v;
             if (next_unit(ln, e2, e2_end, lo2, hi2, MT, v))
                 for (int kb = v.kb0; kb < v.kb1 && kb < v.kb0 + nx.n_stages; ++kb)
-                    tma_prefetch_2d(t.tmW + ln, kb * BK, v.nt * nx.bn);
+                    tma_prefetch_2d(t.tmW + ln, 0, kb * nx.npad + v.nt * nx.bn);
         }
     }
 
@@ -1144,6 +1144,24 @@ made_tc_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ TcDev 
 
 }  // namespace
 
+// Weight layout of this kernel: K-block major, [K block][padded unit][64 inputs], so that the
+// bn x 64 box of one TMA load is one contiguous piece of memory (bn x 128 bytes) instead of bn
+// pieces of 128 bytes a whole weight row apart: a stream of such boxes reads DRAM pages in full.
+__global__ void tile_major_weights(const __nv_bfloat16 *__restrict__ W, __nv_bfloat16 *__restrict__ Wp, int N, int K,
+                                   int npad, int nkb)
+{
+    const size_t total = (size_t)nkb * npad * (BK / 8);
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int j8 = (int)(i % (BK / 8));
+        const size_t rowp = i / (BK / 8);
+        const int n = (int)(rowp % npad), kb = (int)(rowp / npad);
+        const int k = kb * BK + j8 * 8;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (n < N && k < K) v = *reinterpret_cast<const uint4 *>(W + (size_t)n * K + k);     // K is a multiple of 8
+        *reinterpret_cast<uint4 *>(Wp + rowp * BK + j8 * 8) = v;
+    }
+}
+
 // --------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -1257,8 +1275,18 @@ int js_tc_prepare(js_model *mo)
         t.lay[l].n_stages = std::min(MAX_STAGES, ring_cap / t.lay[l].stage_bytes);
         kb_all[l] = kb;
         if (!encode_map(&mapsA[l], v.a[l], mo->rows, K, BM)) return 0;
-        if (!encode_map(&mapsW[l], v.W[l], N, K, bn)) return 0;
+        {
+            const int nkb = (K + BK - 1) / BK, npad = nt * bn;
+            void *wp = nullptr;
+            if (cudaMalloc(&wp, (size_t)nkb * npad * BK * sizeof(__nv_bfloat16)) != cudaSuccess) return JS_ERR_CUDA;
+            mo->allocs.push_back(wp);
+            tile_major_weights<<<1184, 256>>>((const __nv_bfloat16 *)v.W[l], (__nv_bfloat16 *)wp, N, K, npad, nkb);
+            if (cudaGetLastError() != cudaSuccess) return JS_ERR_CUDA;
+            t.lay[l].npad = npad;
+            if (!encode_map(&mapsW[l], wp, nkb * npad, BK, bn)) return 0;
+        }
     }
+    if (cudaDeviceSynchronize() != cudaSuccess) return JS_ERR_CUDA;     // the tile-major copies are complete
     // ---- split-K work units and their static assignment to CTAs (longest processing time first)
     int sms = 0;
     {
