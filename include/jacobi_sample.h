@@ -183,7 +183,8 @@ typedef enum {
     JS_OPT_SPIN_LIMIT = 2,     /* polls before a device-side wait gives up (default 1<<22) */
     JS_OPT_PATH = 3,           /* 0 (default): tensor-core kernels where the model allows; 1: CUDA-core kernels only */
     JS_OPT_COMPACT = 4,        /* 1 (default): move finished samples out of the working batch */
-    JS_OPT_TRACE = 5           /* 0 (default); 1: record device timestamps of the next calls (js_get_trace) */
+    JS_OPT_TRACE = 5           /* 0 (default); 1: record device timestamps of the next calls (js_get_trace) for the
+                                  first and the last CTA; n >= 2: for the first CTA and CTA n - 2 */
 } js_option;
 int js_set_option(js_model *m, int option, int value);
 
@@ -204,7 +205,7 @@ typedef struct {
 int js_get_stats(const js_model *m, js_stats *out);
 
 /* Device-side timeline of the most recent call made with JS_OPT_TRACE on (tensor-core kernels):
- * globaltimer nanoseconds, layout [2][256][12] = [first CTA, last CTA][phase][slot]; a phase is one
+ * globaltimer nanoseconds, layout [2][256][12] = [first CTA, last (or chosen) CTA][phase][slot]; a phase is one
  * layer of one forward pass; slots: 0 phase start, 1 first operands landed, 2 last MMA issued,
  * 3 accumulator complete, 4 epilogue stored, 5 left the grid barrier, 6-11 points inside the
  * epilogue; 0 = not recorded.

@@ -202,6 +202,7 @@ int prep_args(js_model *m, RunArgs &r, cudaStream_t st)
     r.perm_stride = m->rows;
     r.spin_limit = (unsigned)m->opt_spin_limit;
     r.trace = m->opt_trace ? m->trace : nullptr;
+    r.trace_cta = m->opt_trace >= 2 ? m->opt_trace - 2 : -1;
     if (r.trace) CU_TRY(cudaMemsetAsync(m->trace, 0, sizeof(unsigned long long) * 2 * JS_TRACE_PHASES * JS_TRACE_SLOTS, st));
     // a call that ended normally left the control block zeroed
     if (!m->ctl_clean) CU_TRY(cudaMemsetAsync(m->ctl, 0, sizeof(JsCtl), st));
@@ -645,7 +646,7 @@ int js_set_option(js_model *m, int option, int value)
     case JS_OPT_SPIN_LIMIT: if (value < 0) return JS_ERR_ARG; m->opt_spin_limit = value; return JS_OK;
     case JS_OPT_PATH: if (value != 0 && value != 1) return JS_ERR_ARG; m->opt_path = value; return JS_OK;
     case JS_OPT_COMPACT: m->opt_compact = value ? 1 : 0; return JS_OK;
-    case JS_OPT_TRACE: m->opt_trace = value ? 1 : 0; return JS_OK;
+    case JS_OPT_TRACE: m->opt_trace = value > 0 ? value : 0; return JS_OK;
     default: return JS_ERR_ARG;
     }
 }

@@ -85,8 +85,8 @@ struct ConvEngine {
     __device__ void trace(int slot) const
     {
         if (r.trace == nullptr || phase_no >= JS_TRACE_PHASES) return;
-        if (blockIdx.x != 0 && blockIdx.x != gridDim.x - 1) return;
-        const int who = blockIdx.x == 0 ? 0 : 1;
+        const int who = js_trace_who(r);
+        if (who < 0) return;
         r.trace[((size_t)who * JS_TRACE_PHASES + phase_no) * JS_TRACE_SLOTS + slot] = global_ns();
     }
 

@@ -83,7 +83,16 @@ struct RunArgs {
     unsigned noise_stamp;
     JsCtl *result;            // host memory mapped into the device: the last CTA to leave copies ctl here
     unsigned long long *trace;   // [2 CTAs][JS_TRACE_PHASES][JS_TRACE_SLOTS] globaltimer stamps, or NULL
+    int trace_cta;               // the second traced CTA (the first is CTA 0); < 0: the last CTA of the grid
 };
+
+// which of the two traced CTAs this one is (0, 1), or -1
+__device__ __forceinline__ int js_trace_who(const RunArgs &r)
+{
+    if (blockIdx.x == 0) return 0;
+    const unsigned second = r.trace_cta >= 0 && r.trace_cta < (int)gridDim.x ? (unsigned)r.trace_cta : gridDim.x - 1;
+    return blockIdx.x == second ? 1 : -1;
+}
 
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned *p)
 {

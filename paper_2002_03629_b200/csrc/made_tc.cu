@@ -102,8 +102,8 @@ struct TcEngine {
     __device__ void trace(int slot) const
     {
         if (r.trace == nullptr || phase_no >= JS_TRACE_PHASES) return;
-        if (blockIdx.x != 0 && blockIdx.x != gridDim.x - 1) return;
-        const int who = blockIdx.x == 0 ? 0 : 1;
+        const int who = js_trace_who(r);
+        if (who < 0) return;
         r.trace[((size_t)who * JS_TRACE_PHASES + phase_no) * JS_TRACE_SLOTS + slot] = global_ns();
     }
 
@@ -1086,8 +1086,8 @@ made_tc_kernel(const __grid_constant__ MadeDev m, const __grid_constant__ TcDev 
     uint8_t *ring = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
 
     const int warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0 && r.trace != nullptr && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1))
-        r.trace[((size_t)(blockIdx.x == 0 ? 0 : 1) * JS_TRACE_PHASES) * JS_TRACE_SLOTS + 2] = global_ns();   // kernel entry
+    if (threadIdx.x == 0 && r.trace != nullptr && js_trace_who(r) >= 0)
+        r.trace[((size_t)js_trace_who(r) * JS_TRACE_PHASES) * JS_TRACE_SLOTS + 2] = global_ns();   // kernel entry
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&sh.full[s], 1); mbar_init(&sh.empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&sh.tfull[a], 1); mbar_init(&sh.tempty[a], 4); }

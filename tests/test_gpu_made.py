@@ -84,6 +84,10 @@ CHAIN = si.scaled(si.CONFIGS["made_4096"], D=256, H=(256, 256, 256, 256), batch=
 # long K ranges with few tiles: the tensor-core kernels cut every tile's K loop into several work units
 SPLIT = si.scaled(si.CONFIGS["made_784"], D=512, H=(2688, 2688), batch=130, w_var_scale=3.0)
 
+# four row tiles (the last one ragged) and enough 128-wide tiles per hidden layer to go without split K;
+# compaction takes the working batch through every number of row tiles
+ROWS4 = si.scaled(si.CONFIGS["made_784"], D=256, H=(1280, 1280), batch=400, w_var_scale=3.0, index=11)
+
 # more rows than the 256-way epilogue keeps in shared memory: rows beyond load their noise directly
 CAT_ROWS = si.scaled(si.CONFIGS["made_cat"], D=16, H=(64, 64), batch=100)
 
@@ -99,7 +103,7 @@ CAT_ICDF_SPLIT = si.scaled(si.CONFIGS["made_cat"], D=16, H=(2688,), batch=20, no
 CAT7_ICDF = si.MadeConfig("cat7", 9, D=20, C=7, H=(48,), act=si.ACT_RELU, prec=si.PREC_F32, batch=11,
                           noise_kind=si.NOISE_UNIFORM_CAT, w_var_scale=8.0, b_var=0.2)
 
-CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN, "split": SPLIT, "cat_rows": CAT_ROWS,
+CASES = {"tiny": TINY, "bin": BIN, "cat": CAT, "chain": CHAIN, "split": SPLIT, "rows4": ROWS4, "cat_rows": CAT_ROWS,
          "bin_icdf": BIN_ICDF, "cat_icdf": CAT_ICDF, "cat_icdf_split": CAT_ICDF_SPLIT, "cat7_icdf": CAT7_ICDF}
 # kernel path: 1 = CUDA-core kernels, 0 = tensor-core kernels (bf16 models only)
 COMBOS = [(n, 1) for n in CASES] + [(n, 0) for n in CASES if n != "tiny"]

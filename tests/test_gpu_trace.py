@@ -2,7 +2,7 @@
 
 The stamps of a phase must be ordered in time (producer start <= first operands <= last MMA issued,
 last accumulator <= epilogues done <= barrier passed), phases must follow one another, and tracing must
-not change the samples."""
+not change the samples.  The second traced CTA can be chosen."""
 import numpy as np
 import pytest
 import torch
@@ -50,6 +50,17 @@ def test_timeline_is_ordered_and_tracing_changes_nothing(name):
                 assert row[0] <= row[1] <= row[2] <= row[5]
                 assert row[3] <= row[4] <= row[5]
             last_barrier = row[5]
+        # a chosen CTA in the second slot (option value n >= 2 traces CTA n - 2 beside the first one): CTA 1
+        # has a tile in the first phase of both cases, so its row carries a start stamp and a barrier stamp
+        # that lie inside the first CTA's call
+        model.set_option(p.JS_OPT_TRACE, 2 + 1)
+        assert p.jacobi_sample(model, noise, cfg.noise_kind, None, p.JS_JACOBI, 0, 0, out) == 0
+        assert torch.equal(out, ref)
+        both = model.trace().astype(np.int64)
+        first, chosen = both[0], both[1]
+        ph1 = [ph for ph in range(1, first.shape[0]) if first[ph, 5] > 0][0]
+        assert chosen[ph1, 0] > 0 and chosen[ph1, 5] >= chosen[ph1, 0]
+        assert abs(chosen[ph1, 5] - first[ph1, 5]) < 1_000_000          # the same barrier, within a millisecond
         model.set_option(p.JS_OPT_TRACE, 0)
     finally:
         model.close()
