@@ -20,8 +20,8 @@ constexpr int KC = 32;         // k chunk staged in shared memory
 constexpr int NTHREADS = 256;
 
 struct Smem {
-    float As[KC][GT + 4];
-    float Bs[KC][GT + 4];
+    alignas(16) float As[KC][GT + 4];       // read as float4: rows of GT + 4 floats keep every group of four on 16 bytes
+    alignas(16) float Bs[KC][GT + 4];
     int list[4096];            // Jacobi-GS: units to evaluate in this micro-step
     int list_n;
     int wcnt[NTHREADS / 32];
@@ -38,28 +38,41 @@ __device__ void gemm_tile(Smem &s, const T *A, int lda, const T *__restrict__ W,
     for (int i = 0; i < 4; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = 0.0f;
-    for (int k0 = 0; k0 < kend; k0 += KC) {
+    // the operands of the next K step are fetched into registers while the current one is multiplied
+    // (the sums themselves are taken in the same order as without the prefetch)
+    constexpr int PER = (GT * KC) / NTHREADS;
+    float av[PER], bv[PER];
+    auto fetch = [&](int k0) {
 #pragma unroll
-        for (int it = 0; it < (GT * KC) / NTHREADS; ++it) {
+        for (int it = 0; it < PER; ++it) {
             const int idx = tid + it * NTHREADS;
             const int kk = idx % KC, row = idx / KC;
             const int k = k0 + kk;
-            float av = 0.0f, bv = 0.0f;
+            av[it] = 0.0f;
+            bv[it] = 0.0f;
             if (k < kend) {
-                if (m0 + row < M) av = to_f32<T>(A[(size_t)(m0 + row) * lda + k]);
-                if (n0 + row < N) bv = to_f32<T>(W[(size_t)(n0 + row) * ldw + k]);
+                if (m0 + row < M) av[it] = to_f32<T>(A[(size_t)(m0 + row) * lda + k]);
+                if (n0 + row < N) bv[it] = to_f32<T>(W[(size_t)(n0 + row) * ldw + k]);
             }
-            s.As[kk][row] = av;
-            s.Bs[kk][row] = bv;
+        }
+    };
+    if (kend > 0) fetch(0);
+    for (int k0 = 0; k0 < kend; k0 += KC) {
+#pragma unroll
+        for (int it = 0; it < PER; ++it) {
+            const int idx = tid + it * NTHREADS;
+            const int kk = idx % KC, row = idx / KC;
+            s.As[kk][row] = av[it];
+            s.Bs[kk][row] = bv[it];
         }
         __syncthreads();
+        if (k0 + KC < kend) fetch(k0 + KC);
 #pragma unroll 8
         for (int kk = 0; kk < KC; ++kk) {
-            float a[4], b[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) a[i] = s.As[kk][ty * 4 + i];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) b[j] = s.Bs[kk][tx * 4 + j];
+            // (rows of As / Bs are GT + 4 floats: every row and every group of four starts on 16 bytes)
+            const float4 a4 = *reinterpret_cast<const float4 *>(&s.As[kk][ty * 4]);
+            const float4 b4 = *reinterpret_cast<const float4 *>(&s.Bs[kk][tx * 4]);
+            const float a[4] = {a4.x, a4.y, a4.z, a4.w}, b[4] = {b4.x, b4.y, b4.z, b4.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i)
 #pragma unroll
