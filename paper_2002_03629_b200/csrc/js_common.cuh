@@ -116,6 +116,7 @@ __device__ __forceinline__ bool grid_barrier(JsCtl *ctl, unsigned &epoch, unsign
 {
     __syncthreads();
     epoch += 1;
+    if (gridDim.x == 1) return true;      // a single CTA: the block-wide barrier above is all there is to wait for
     int ok = 1;
     if (threadIdx.x == 0) {
         const unsigned target = epoch * gridDim.x;
